@@ -1,0 +1,83 @@
+/*
+ * CPU oracle for DaSGD (Local SGD with Delayed Averaging) -- TEST INFRASTRUCTURE.
+ *
+ * A plain, slow, single-pass restatement of the paper's update rule, used only to
+ * check other implementations.  It is not a product code path and nothing in the
+ * library may call it.  It shares no code with the CUDA implementation.
+ *
+ * What it follows:
+ *   - Local step: Eq. 2, "otherwise" branch (Section III-C-1; restated in
+ *     Appendix "Update Rule"):  x <- x - eta * g(x).  Momentum and weight decay are
+ *     only named as hyper-parameters in Section IV-A ("weight decay 0.01, moment
+ *     0.9"); the formula used is the usual one of the paper's platform:
+ *     g' = g + lambda*w;  m <- mu*m + g' (m_0 = 0);  w <- w - eta*m.
+ *   - Snapshot: the bracketed term of Eq. 2, second branch: each worker's weights
+ *     right after the local step that closes a tau-block (Fig. 2 narrative:
+ *     "after 3 local updates" for tau = 3).
+ *   - Worker-axis mean: the (1/M) * sum_j of Eq. 2 (right-multiplication by J in
+ *     the matrix form of Appendix "Matrix Representation").
+ *   - Delayed merge: Eq. 2, second branch, appendix condition (k+1-d) mod tau = 0:
+ *     x <- xi*(x - eta*g) + (1-xi)*mean, i.e. a xi-blend applied to the already
+ *     locally-stepped weights, d steps after the snapshot.
+ *   - A second merge form, w <- w + (mean - snapshot_of_this_worker), is provided
+ *     as merge_mode 1.  It is NOT in the paper.
+ *
+ * Numerics: state (w, m, snapshot, mean) is float32; every element is computed in
+ * double from the float32 state and rounded to float32 once, at the store.  In
+ * dtype 1 gradients arrive as bfloat16 (widened exactly) and a bfloat16 copy of
+ * the weights, rounded to nearest-even, is refreshed after every write of w.
+ *
+ * Pins (tests marked "not gpu"): hand-worked trajectories derived from Eq. 2,
+ * the minibatch-SGD and Local-SGD special cases (Eq. 1, Section II-C-3), the
+ * averaged-model recursion of Section III-C-1, the deviation contraction used in
+ * the proof of the theorem (Appendix), closed forms for momentum and weight
+ * decay, torch.optim.SGD for the momentum/weight-decay local step, and torch's
+ * bfloat16 cast for the rounding.
+ * Parity unpinned by the paper: schedules with d > tau (the paper assumes
+ * d <= tau) -- defined here by pipelining snapshots, checked by invariants only.
+ */
+#ifndef DASGD_ORACLE_H
+#define DASGD_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct oracle_dasgd oracle_dasgd;
+
+enum { ORACLE_F32 = 0, ORACLE_BF16_MASTER_F32 = 1 };
+enum { ORACLE_MERGE_XI = 0, ORACLE_MERGE_DELTA = 1 };
+enum { ORACLE_OK = 0, ORACLE_ERR_ARG = 1, ORACLE_ERR_STATE = 2 };
+
+/* K workers, P parameters, period tau >= 1, delay d >= 0, blend xi in [0,1]. */
+oracle_dasgd *oracle_dasgd_create(int32_t K, int64_t P, int32_t tau, int32_t d, float xi,
+                                  float momentum, float weight_decay, int32_t dtype,
+                                  int32_t merge_mode);
+void oracle_dasgd_destroy(oracle_dasgd *o);
+
+/* State access: w, m are [K][P] float32 (row k = worker k); w_lp is [K][P] bf16 bits. */
+int oracle_dasgd_set_state(oracle_dasgd *o, const float *w, const float *m);
+int oracle_dasgd_get_state(const oracle_dasgd *o, float *w, float *m, uint16_t *w_lp);
+int64_t oracle_dasgd_steps_done(const oracle_dasgd *o);
+int32_t oracle_dasgd_pending(const oracle_dasgd *o);
+/* mean / snapshot of the i-th oldest pending snapshot (0 = oldest); either may be NULL */
+int oracle_dasgd_get_pending(const oracle_dasgd *o, int32_t i, int64_t *s, float *snap,
+                             float *mean);
+
+/* The four operations of the path; g is [K][P] float32 (dtype 0) or bf16 bits (dtype 1). */
+int oracle_dasgd_local_step(oracle_dasgd *o, const void *g, float lr);
+int oracle_dasgd_snapshot(oracle_dasgd *o);
+int oracle_dasgd_average(oracle_dasgd *o); /* mean of the oldest snapshot not yet averaged */
+int oracle_dasgd_merge(oracle_dasgd *o);   /* blend the OLDEST pending mean, then drop it   */
+
+/* One iteration of the schedule: local step; merge if one lands; snapshot+mean if due. */
+int oracle_dasgd_step(oracle_dasgd *o, const void *g, float lr);
+
+int oracle_dasgd_threads(void); /* OpenMP threads the element loops use (1 if built without) */
+
+#ifdef __cplusplus
+}
+#endif
+#endif
