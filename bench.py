@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the DaSGD hot path (local step + snapshot + worker-axis mean + delayed merge).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload resnet50|small]
+
+One "step" is one pass of the whole path over one batch of synthetic gradients: a local step of
+all K replicas, the merge that lands on that step, the snapshot and the side-stream mean.
+Workload "resnet50": K=8 replicas of a P=25.6M float32 vector, momentum 0.9, weight decay 1e-4,
+lr 0.1, tau=1, d=1, xi=0.25.  Prints ONE JSON line (rank 0).
+
+--impl reference times the plain CPU checker under oracle/ on the host cores, on a bounded slice of
+the same workload (the path is independent across the parameter index, so a slice is exact).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2006_00441_b200 import inputs  # noqa: E402
+
+WORKLOADS = {
+    # name: K, P, momentum, weight_decay, lr, tau, d, xi, grad std, w0 std
+    "resnet50": dict(K=8, P=25_600_000, momentum=0.9, weight_decay=1e-4, lr=0.1, tau=1, d=1, xi=0.25,
+                     g_std=1e-3 ** 0.5, w_std=0.02),
+    "small": dict(K=4, P=1024, momentum=0.0, weight_decay=0.0, lr=0.01, tau=4, d=1, xi=0.25,
+                  g_std=1.0, w_std=0.0),
+}
+METRIC = "replica-param updates/s"
+UNIT = "updates/s"
+RING = 4                       # gradient buffers resident in HBM, used round-robin
+BYTES_PER_UPDATE_STEP = 20     # local step, float32 + momentum: read w, m, g; write w, m
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc, self.path = None, None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            ident = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", ident, f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0])); mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = max(mx)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+
+def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmup: int = 0):
+    """Times the CPU checker on the first P_s parameters of every replica.  Returns a dict."""
+    import numpy as np
+
+    import oracle
+
+    K = wl["K"]
+    probe = oracle.OracleDaSGD(K, 1, 1, 1, 0.5, omp=True)
+    cores = probe.threads
+    probe.close()
+    # calibrate on a slice too large for the CPU caches, so the rate is the DRAM-bound one
+    Pc = min(wl["P"], 2_000_000)
+    o = oracle.OracleDaSGD(K, Pc, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], omp=True)
+    o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=range(Pc)).numpy())
+    g = inputs.grad_block(0, 0, K, wl["P"], wl["g_std"], p_index=range(Pc)).numpy()
+    for _ in range(2):
+        o.step(g, wl["lr"])
+    t0 = time.perf_counter()
+    n_cal = 5
+    for _ in range(n_cal):
+        o.step(g, wl["lr"])
+    rate = K * Pc * n_cal / (time.perf_counter() - t0)  # updates/s, rough
+    o.close()
+    if steps is None:       # cpu_baseline leg: fixed slice, as many steps as fit the budget
+        Ps = min(wl["P"], 2_000_000)
+        steps = max(3, min(200, int(seconds_budget * rate / (K * Ps))))
+    else:                   # reference arm: the caller fixes the steps, the slice is sized to the budget
+        Ps = int(min(wl["P"], 4_000_000, max(1024, seconds_budget * rate / (K * (steps + warmup)))))
+    idx = range(Ps)
+    o = oracle.OracleDaSGD(K, Ps, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], omp=True)
+    o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=idx).numpy())
+    ring = [inputs.grad_block(0, t, K, wl["P"], wl["g_std"], p_index=idx).numpy() for t in range(2)]
+    for t in range(warmup):
+        o.step(ring[t % 2], wl["lr"])
+    t0 = time.perf_counter()
+    for t in range(steps):
+        o.step(ring[t % 2], wl["lr"])
+    dt = time.perf_counter() - t0
+    assert np.isfinite(o.w).all()
+    o.close()
+    return {"value": K * Ps * steps / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {Ps} of {wl['P']} parameters of all {K} replicas, {steps} steps "
+                      f"(OpenMP build of the checker, {cores} threads)",
+            "seconds": dt, "steps": steps, "P_sample": Ps}
+
+
+def run_reference(args, wl, name):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    r = oracle_throughput(wl, seconds_budget=60.0, steps=args.steps, warmup=args.warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * r["seconds"] / r["steps"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(wl, name),
+        "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl, name):
+    return {"workload": f"{name}: K={wl['K']} replicas x P={wl['P']} float32, momentum {wl['momentum']}, "
+                        f"weight decay {wl['weight_decay']}, lr {wl['lr']}, tau={wl['tau']}, d={wl['d']}, xi={wl['xi']}",
+            "K": wl["K"], "P": wl["P"], "tau": wl["tau"], "d": wl["d"], "xi": wl["xi"],
+            "l2_policy": "inputs larger than L2 (each step streams K*P*20 B; gradient ring of 4 buffers)",
+            "parallelism": "independent replicas of the workload per GPU (no collective on this path)"}
+
+
+# ------------------------------------------------------------------ our arm
+
+def run_ours(args, wl, name):
+    from paper_2006_00441_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K, P, lr = wl["K"], wl["P"], wl["lr"]
+    flags_fused = B.DASGD_FLAG_FUSE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE
+    seed = 1000 + rank  # every rank runs its own replica of the workload
+
+    def make(flags, host_staging=False):
+        e = B.DaSGD(K, P, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], flags=flags,
+                    device=local_rank, host_staging=host_staging, order_after_current=False)
+        e.set_state(inputs.shared_start(seed, P, wl["w_std"], device="cuda"))
+        return e
+
+    ring = [inputs.grad_block(seed, t, K, P, wl["g_std"], device="cuda") for t in range(RING)]
+    torch.cuda.synchronize()
+
+    def timed_loop(e, steps, warmup, step_fn):
+        for t in range(warmup):
+            step_fn(e, t)
+        e.sync()
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = e.launches
+        with torch.cuda.stream(e.main):
+            ev0.record()
+        for t in range(steps):
+            step_fn(e, warmup + t)
+        e.main.wait_stream(e.side)        # the last mean belongs to the timed work
+        with torch.cuda.stream(e.main):
+            ev1.record()
+        e.sync()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if dist is not None:
+            tms = torch.tensor([ms], device="cuda")
+            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+            ms = float(tms.item())
+        return ms, e.launches - l0
+
+    def dev_step(e, t):
+        e.step(ring[t % RING], lr)
+
+    # ---- headline: inputs resident in HBM
+    eng = make(flags_fused)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms, launches = timed_loop(eng, args.steps, args.warmup, dev_step)
+    clocks = sampler.stop() if sampler else None
+    value = world * K * P * args.steps / (ms * 1e-3)
+    eng.close()
+    del eng
+
+    # ---- instrumented pass: per-kernel device time and the hidden fraction of the averaging
+    eng = make(flags_fused | B.DASGD_FLAG_TIMING)
+    for t in range(args.warmup):
+        dev_step(eng, t)
+    eng.reset_timing()
+    n_inst = min(args.steps, 100)
+    for t in range(n_inst):
+        dev_step(eng, args.warmup + t)
+    kt = eng.kernel_timing()
+    eng.close()
+    del eng
+    peak, peak_kind = measured_peak_gbs()
+    n_step, ms_step = kt["local_step"]
+    step_gbs = (K * P * BYTES_PER_UPDATE_STEP / 1e9) / (ms_step / n_step * 1e-3) if n_step else None
+    hidden = None
+    if kt["mean"][0] and kt["mean"][1] > 0:
+        hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
+
+    # ---- end to end: gradients start in page-locked host memory every step
+    e2e = None
+    try:
+        eng = make(flags_fused, host_staging=True)
+        hosts = [torch.empty((K, P), dtype=torch.float32).pin_memory() for _ in range(2)]
+        for i, h in enumerate(hosts):
+            h.copy_(ring[i])
+        probe = torch.empty(1024, dtype=torch.float32).pin_memory()
+        torch.cuda.synchronize()
+        e2e_steps = max(3, min(args.steps, 20))
+
+        def host_step(e, t):
+            e.step_host(hosts[t % 2], lr, probe)
+
+        ms_e, _ = timed_loop(eng, e2e_steps, 3, host_step)
+        e2e = {"value": world * K * P * e2e_steps / (ms_e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": K * P * 4, "d2h_bytes_per_step": probe.numel() * 4,
+               "steps": e2e_steps, "ms_per_step": ms_e / e2e_steps}
+        eng.close()
+        del eng, hosts
+    except Exception as ex:  # page-locked memory can be refused on a small host
+        e2e = {"value": None, "unit": UNIT, "error": str(ex)[:200]}
+
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+
+    cpu = oracle_throughput(wl, seconds_budget=15.0)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": workload_config(wl, name),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "k_local_step_vec (float32, momentum)",
+                     "achieved": step_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": (step_gbs / peak) if step_gbs else None, "peak_kind": f"of {peak_kind}",
+                     "frac_of_8TBs": (step_gbs / 8000.0) if step_gbs else None,
+                     "algorithmic_bytes_per_launch": K * P * BYTES_PER_UPDATE_STEP,
+                     "avg_launch_ms": (ms_step / n_step) if n_step else None,
+                     "timed": f"CUDA events on the launching stream, instrumented pass of {n_inst} steps",
+                     "traffic": None},
+        "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
+        "averaging_hidden_frac": hidden,
+        "whole_path_gbs": value / world * path_bytes_per_update(wl) / 1e9,
+        "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def path_bytes_per_update(wl):
+    """Algorithmic HBM bytes per replica-parameter update of the whole path as scheduled with both
+    fusion flags, float32 + momentum: tau local steps (20 B each), the snapshot stored by the kernel
+    that last writes w (4 B), the mean (4 + 4/K B), and the merge (4/K B inside a step kernel when
+    d >= 2, else a pass of its own: 8 + 4/K B)."""
+    K, tau, d = wl["K"], wl["tau"], wl["d"]
+    per_cycle = 20.0 * tau + 4.0 + (4.0 + 4.0 / K)
+    per_cycle += (4.0 / K) if d >= 2 else (8.0 + 4.0 / K)
+    return per_cycle / tau
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl, args.workload)
+    else:
+        run_ours(args, wl, args.workload)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,169 @@
+/*
+ * libdasgd -- DaSGD (Local SGD with Delayed Averaging) hot path for NVIDIA B200 (sm_100a).
+ *
+ * K worker replicas of a P-element model live as rows of [K][ld] arrays in one GPU's memory
+ * (ld >= P is the row stride in elements).  The library applies, with hand-written CUDA kernels,
+ *   - the local step of every worker          (Eq. 2, "otherwise" branch, Section III-C-1),
+ *   - the snapshot of the just-stepped weights (the bracketed term of Eq. 2's second branch),
+ *   - the mean over the worker axis            (the (1/M)*sum_j of Eq. 2; "J" in the Appendix),
+ *   - the delayed merge                        (Eq. 2, second branch),
+ * and schedules the mean on a side stream so that it runs while the next local steps proceed
+ * (the overlap of Section III, Fig. 2, and of Eq. 6's condition t_c < d*t_p).
+ *
+ * Conventions
+ *   - Every pointer named "device" is a CUDA device pointer on the context's device; every
+ *     pointer named "host" is ordinary (preferably page-locked) host memory.
+ *   - All device buffers and both streams are owned by the caller and must stay valid until
+ *     dasgd_destroy().  The library owns only its host-side context and its CUDA events.
+ *   - All calls are asynchronous with respect to the host except dasgd_sync, dasgd_get_timing
+ *     and dasgd_destroy.  A context is not thread-safe; different contexts are independent.
+ *   - Every call returns a dasgd_status and never aborts.  After a non-OK status
+ *     dasgd_last_error() gives a one-line explanation.
+ *   - Step counting: t = number of completed local steps.  Snapshots are taken when t is a
+ *     positive multiple of tau; the snapshot taken at t = s is merged when t = s + d
+ *     (Appendix form of the condition, (k+1-d) mod tau = 0; Fig. 2 for the indexing).
+ */
+#ifndef DASGD_H
+#define DASGD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dasgd_ctx dasgd_ctx;
+
+typedef enum {
+  DASGD_OK = 0,
+  DASGD_ERR_INVALID_ARG = 1,   /* bad configuration or NULL / misaligned pointer            */
+  DASGD_ERR_BAD_STATE = 2,     /* call out of order (nothing to average, nothing to merge)   */
+  DASGD_ERR_NO_SLOT = 3,       /* snapshot requested while every slot holds a pending average */
+  DASGD_ERR_CUDA = 4,          /* a CUDA runtime call failed; see dasgd_last_error            */
+  DASGD_ERR_TIMEOUT = 5,       /* dasgd_sync gave up waiting                                  */
+  DASGD_ERR_UNSUPPORTED = 6    /* valid request this build cannot serve                       */
+} dasgd_status;
+
+typedef enum {
+  DASGD_F32 = 0,            /* gradients, weights, momentum: float32                                   */
+  DASGD_BF16_MASTER_F32 = 1 /* gradients bfloat16; float32 master weights + momentum; a bfloat16 copy
+                               of the weights (w_lp) is rewritten, round-to-nearest-even, with every
+                               write of the master                                                    */
+} dasgd_dtype;
+
+typedef enum {
+  DASGD_MERGE_XI = 0,   /* w_k <- xi*w_k + (1-xi)*mean          (Eq. 2, second branch)                 */
+  DASGD_MERGE_DELTA = 1 /* w_k <- w_k + (mean - snapshot_k)     (not in the paper; keeps local progress) */
+} dasgd_merge_mode;
+
+/* flags */
+#define DASGD_FLAG_TIMING 0x1u        /* record CUDA events around every average and every wait for it */
+#define DASGD_FLAG_FUSE_SNAPSHOT 0x2u /* dasgd_step: store the snapshot from the kernel that last writes
+                                         w in that step instead of running a separate copy             */
+#define DASGD_FLAG_FUSE_MERGE 0x4u    /* dasgd_step: when d >= 2, blend the mean inside the local-step
+                                         kernel of the step the merge lands on                         */
+
+typedef struct dasgd_config {
+  int32_t K;            /* workers (the paper's M), >= 1                                              */
+  int32_t tau;          /* local steps between snapshots, >= 1                                        */
+  int32_t d;            /* delay in local steps between snapshot and merge, >= 0 (0 = Local SGD)      */
+  int32_t dtype;        /* dasgd_dtype                                                                */
+  int32_t merge_mode;   /* dasgd_merge_mode                                                           */
+  int32_t n_slots;      /* snapshot/mean slots provided; must be >= max(1, ceil(d/tau))               */
+  uint32_t flags;       /* DASGD_FLAG_*                                                               */
+  int32_t device;       /* CUDA device ordinal that owns every buffer and both streams                */
+  int64_t P;            /* parameters per worker, >= 1                                                */
+  int64_t ld;           /* row stride in elements of every [K][ld] array; 0 means P.  Rows start on
+                           16-byte boundaries (full-speed path) when ld % 8 == 0                      */
+  float xi;             /* local proportion in the merge, 0 <= xi <= 1                                */
+  float momentum;       /* mu; 0 disables the momentum buffer (m may then be NULL)                    */
+  float weight_decay;   /* lambda, coupled L2: g' = g + lambda*w                                      */
+  uint32_t sync_timeout_ms; /* dasgd_sync gives up after this long; 0 means 60000                     */
+  void *w;              /* device, [K][ld] float32, in/out: weights (master weights in bf16 mode)     */
+  void *m;              /* device, [K][ld] float32, in/out: momentum buffers (start them at 0)        */
+  void *w_lp;           /* device, [K][ld] bfloat16, out: low-precision weights; bf16 mode only       */
+  void *snap;           /* device, [n_slots][K][ld] float32, scratch: snapshots                       */
+  void *mean;           /* device, [n_slots][ld] float32, scratch: worker-axis means                  */
+  void *g_stage;        /* device, [K][ld] gradient dtype, scratch for dasgd_step_host; may be NULL   */
+  void *main_stream;    /* cudaStream_t carrying local steps, snapshots and merges                    */
+  void *side_stream;    /* cudaStream_t carrying the averages; must differ from main_stream           */
+} dasgd_config;
+
+/* Validates cfg, copies it, creates the events.  No kernel is launched.  *out is NULL on error
+ * (the error text is then available from dasgd_last_error(NULL)). */
+dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg);
+
+/* Local step for all K workers on the main stream (Eq. 2 first branch; momentum / weight decay in
+ * the usual form of Section IV-A's hyper-parameters):
+ *     g' = g + lambda*w;   m <- mu*m + g';   w <- w - lr*m        (mu == 0: w <- w - lr*g')
+ * grads: device, [K][ld], float32 or bfloat16 according to dtype; read only; must stay untouched
+ * until the main stream has passed this call.  Increments t. */
+dasgd_status dasgd_local_step(dasgd_ctx *ctx, const void *grads_device, float lr);
+
+/* Main stream: copy w into a free slot (Eq. 2: the quantity that is averaged).  DASGD_ERR_NO_SLOT if
+ * every slot still holds a pending average. */
+dasgd_status dasgd_snapshot(dasgd_ctx *ctx);
+
+/* Side stream: mean over the K rows of the oldest snapshot that has none yet.  Returns at once;
+ * the main stream is not blocked.  DASGD_ERR_BAD_STATE if no such snapshot exists. */
+dasgd_status dasgd_average_async(dasgd_ctx *ctx);
+
+/* Main stream: wait (on the device) for the OLDEST pending average, blend it into every worker's
+ * current weights according to merge_mode, release the slot.  DASGD_ERR_BAD_STATE if no average is
+ * pending.  This wait is the only point where averaging can delay local work. */
+dasgd_status dasgd_merge(dasgd_ctx *ctx);
+
+/* Host waits (bounded by sync_timeout_ms) until both streams have drained; reports CUDA errors
+ * raised by earlier asynchronous work.  Pending averages stay pending; nothing is applied. */
+dasgd_status dasgd_sync(dasgd_ctx *ctx);
+
+/* One iteration of the schedule, all asynchronous:
+ *     local step;  if a snapshot from t-d is due, merge it;  if t % tau == 0, snapshot + average
+ * (d == 0: snapshot, average and merge in the same iteration, i.e. Local SGD).  Honors the
+ * FUSE flags; results are the same with and without them. */
+dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads_device, float lr);
+
+/* dasgd_step for callers whose gradients are in HOST memory: copies grads_host ([K][ld], gradient
+ * dtype) into cfg.g_stage on the main stream, runs dasgd_step, and, if probe_host != NULL, copies
+ * the first probe_elems float32 weights of worker 0 back into probe_host.  Both host buffers must
+ * stay valid until the main stream has passed this call (page-locked memory keeps the copies
+ * asynchronous).  DASGD_ERR_BAD_STATE if cfg.g_stage was NULL. */
+dasgd_status dasgd_step_host(dasgd_ctx *ctx, const void *grads_host, float lr, float *probe_host,
+                             int64_t probe_elems);
+
+/* t, the number of completed local steps, and the number of snapshots awaiting their merge. */
+dasgd_status dasgd_get_step(const dasgd_ctx *ctx, int64_t *t, int32_t *pending);
+
+/* Device pointers of the i-th oldest pending slot (0 = oldest) and the step it was taken at. */
+dasgd_status dasgd_get_pending(const dasgd_ctx *ctx, int32_t i, int64_t *s, void **snap_device,
+                               void **mean_device);
+
+/* Requires DASGD_FLAG_TIMING.  Synchronises, then returns sums over all averages completed since
+ * the last dasgd_reset_timing: n_avg averages, ms_avg = time the averaging kernels took on the side stream,
+ * ms_stall = time the main stream spent waiting for them before merges.  The fraction of
+ * averaging hidden behind local work is 1 - ms_stall/ms_avg (Section V, Eq. 6). */
+dasgd_status dasgd_get_timing(dasgd_ctx *ctx, int64_t *n_avg, double *ms_avg, double *ms_stall);
+
+/* Requires DASGD_FLAG_TIMING.  Synchronises, then returns the number of launches and the summed
+ * device time (CUDA events on the launching stream) of one kind of work since the last
+ * dasgd_reset_timing: which = 0 local-step kernels (fused variants included), 1 snapshot copies,
+ * 2 worker-axis means, 3 merge kernels, 4 the main stream's waits for a mean. */
+dasgd_status dasgd_get_kernel_timing(dasgd_ctx *ctx, int32_t which, int64_t *n, double *ms);
+
+/* Synchronises and zeroes every timing counter. */
+dasgd_status dasgd_reset_timing(dasgd_ctx *ctx);
+
+/* Number of kernels this context has launched so far. */
+dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches);
+
+const char *dasgd_strerror(dasgd_status s);
+const char *dasgd_last_error(const dasgd_ctx *ctx); /* ctx may be NULL: last dasgd_init failure */
+dasgd_status dasgd_destroy(dasgd_ctx *ctx);         /* synchronises both streams, frees the context */
+
+/* Library version, "major.minor". */
+const char *dasgd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,311 @@
+"""ctypes binding of libdasgd.so: argument marshalling only.
+
+Every step of the path (local step, snapshot, worker-axis mean, merge, scheduling) runs inside
+the native library; torch is used here for device memory and streams.  If the library cannot be
+loaded the import fails -- there is no other implementation to fall back to.
+
+The module-level ``dasgd_*`` functions mirror the C ABI of ``include/dasgd.h`` one to one
+(raising ``DasgdError`` on a non-OK status); ``DaSGD`` is a small convenience wrapper that
+allocates the caller-owned buffers as torch tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+
+import torch
+
+from . import build as _build
+
+# ---------------------------------------------------------------- constants (include/dasgd.h)
+DASGD_OK, DASGD_ERR_INVALID_ARG, DASGD_ERR_BAD_STATE, DASGD_ERR_NO_SLOT = 0, 1, 2, 3
+DASGD_ERR_CUDA, DASGD_ERR_TIMEOUT, DASGD_ERR_UNSUPPORTED = 4, 5, 6
+DASGD_F32, DASGD_BF16_MASTER_F32 = 0, 1
+DASGD_MERGE_XI, DASGD_MERGE_DELTA = 0, 1
+DASGD_FLAG_TIMING, DASGD_FLAG_FUSE_SNAPSHOT, DASGD_FLAG_FUSE_MERGE = 0x1, 0x2, 0x4
+
+EXPORTS = [
+    "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
+    "dasgd_step", "dasgd_step_host", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
+    "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
+]
+
+
+class dasgd_config(ctypes.Structure):
+    _fields_ = [
+        ("K", ctypes.c_int32), ("tau", ctypes.c_int32), ("d", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("merge_mode", ctypes.c_int32), ("n_slots", ctypes.c_int32), ("flags", ctypes.c_uint32),
+        ("device", ctypes.c_int32), ("P", ctypes.c_int64), ("ld", ctypes.c_int64),
+        ("xi", ctypes.c_float), ("momentum", ctypes.c_float), ("weight_decay", ctypes.c_float),
+        ("sync_timeout_ms", ctypes.c_uint32),
+        ("w", ctypes.c_void_p), ("m", ctypes.c_void_p), ("w_lp", ctypes.c_void_p), ("snap", ctypes.c_void_p),
+        ("mean", ctypes.c_void_p), ("g_stage", ctypes.c_void_p),
+        ("main_stream", ctypes.c_void_p), ("side_stream", ctypes.c_void_p),
+    ]
+
+
+class DasgdError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"libdasgd status {status}: {text}")
+        self.status = status
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()  # raises if nvcc is unavailable
+    L = ctypes.CDLL(path)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    L.dasgd_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(dasgd_config)]
+    L.dasgd_local_step.argtypes = [vp, vp, f32]
+    L.dasgd_snapshot.argtypes = [vp]
+    L.dasgd_average_async.argtypes = [vp]
+    L.dasgd_merge.argtypes = [vp]
+    L.dasgd_sync.argtypes = [vp]
+    L.dasgd_step.argtypes = [vp, vp, f32]
+    L.dasgd_step_host.argtypes = [vp, vp, f32, vp, i64]
+    L.dasgd_get_step.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i32)]
+    L.dasgd_get_pending.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    L.dasgd_get_timing.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double),
+                                   ctypes.POINTER(ctypes.c_double)]
+    L.dasgd_get_launches.argtypes = [vp, ctypes.POINTER(i64)]
+    L.dasgd_get_kernel_timing.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.dasgd_reset_timing.argtypes = [vp]
+    L.dasgd_strerror.argtypes = [ctypes.c_int]
+    L.dasgd_strerror.restype = ctypes.c_char_p
+    L.dasgd_last_error.argtypes = [vp]
+    L.dasgd_last_error.restype = ctypes.c_char_p
+    L.dasgd_destroy.argtypes = [vp]
+    L.dasgd_version.argtypes = []
+    L.dasgd_version.restype = ctypes.c_char_p
+    return L
+
+
+_L = _load()
+
+
+def _check(status: int, ctx=None):
+    if status != DASGD_OK:
+        detail = _L.dasgd_last_error(ctx).decode() if (ctx or status) else ""
+        raise DasgdError(status, f"{_L.dasgd_strerror(status).decode()}: {detail}")
+
+
+# ---------------------------------------------------------------- the C ABI, name for name
+
+def dasgd_version() -> str:
+    return _L.dasgd_version().decode()
+
+
+def dasgd_init(cfg: dasgd_config) -> ctypes.c_void_p:
+    ctx = ctypes.c_void_p()
+    _check(_L.dasgd_init(ctypes.byref(ctx), ctypes.byref(cfg)), None)
+    return ctx
+
+
+def dasgd_local_step(ctx, grads_ptr: int, lr: float):
+    _check(_L.dasgd_local_step(ctx, grads_ptr, lr), ctx)
+
+
+def dasgd_snapshot(ctx):
+    _check(_L.dasgd_snapshot(ctx), ctx)
+
+
+def dasgd_average_async(ctx):
+    _check(_L.dasgd_average_async(ctx), ctx)
+
+
+def dasgd_merge(ctx):
+    _check(_L.dasgd_merge(ctx), ctx)
+
+
+def dasgd_sync(ctx):
+    _check(_L.dasgd_sync(ctx), ctx)
+
+
+def dasgd_step(ctx, grads_ptr: int, lr: float):
+    _check(_L.dasgd_step(ctx, grads_ptr, lr), ctx)
+
+
+def dasgd_step_host(ctx, grads_host_ptr: int, lr: float, probe_host_ptr: int | None, probe_elems: int):
+    _check(_L.dasgd_step_host(ctx, grads_host_ptr, lr, probe_host_ptr, probe_elems), ctx)
+
+
+def dasgd_get_step(ctx):
+    t, pend = ctypes.c_int64(), ctypes.c_int32()
+    _check(_L.dasgd_get_step(ctx, ctypes.byref(t), ctypes.byref(pend)), ctx)
+    return t.value, pend.value
+
+
+def dasgd_get_pending(ctx, i: int):
+    s, snap, mean = ctypes.c_int64(), ctypes.c_void_p(), ctypes.c_void_p()
+    _check(_L.dasgd_get_pending(ctx, i, ctypes.byref(s), ctypes.byref(snap), ctypes.byref(mean)), ctx)
+    return s.value, snap.value, mean.value
+
+
+def dasgd_get_timing(ctx):
+    n, a, st = ctypes.c_int64(), ctypes.c_double(), ctypes.c_double()
+    _check(_L.dasgd_get_timing(ctx, ctypes.byref(n), ctypes.byref(a), ctypes.byref(st)), ctx)
+    return n.value, a.value, st.value
+
+
+def dasgd_get_kernel_timing(ctx, which: int):
+    n, ms = ctypes.c_int64(), ctypes.c_double()
+    _check(_L.dasgd_get_kernel_timing(ctx, which, ctypes.byref(n), ctypes.byref(ms)), ctx)
+    return n.value, ms.value
+
+
+def dasgd_reset_timing(ctx):
+    _check(_L.dasgd_reset_timing(ctx), ctx)
+
+
+def dasgd_get_launches(ctx) -> int:
+    n = ctypes.c_int64()
+    _check(_L.dasgd_get_launches(ctx, ctypes.byref(n)), ctx)
+    return n.value
+
+
+def dasgd_destroy(ctx):
+    _check(_L.dasgd_destroy(ctx), None)
+
+
+# ---------------------------------------------------------------- convenience wrapper
+
+def min_slots(tau: int, d: int) -> int:
+    return max(1, math.ceil(d / tau))
+
+
+class DaSGD:
+    """K replicas of a P-vector on one GPU.  Owns the torch tensors and streams the library borrows.
+
+    ``w``, ``m`` are ``[K, ld]`` float32 tensors (``[:, :P]`` is the payload); in bf16 mode ``w_lp``
+    is the ``[K, ld]`` bfloat16 copy.  ``main`` / ``side`` are the two torch streams.
+    """
+
+    def __init__(self, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=DASGD_F32,
+                 merge_mode=DASGD_MERGE_XI, flags=0, n_slots=None, ld=None, device=0, host_staging=False,
+                 sync_timeout_ms=0, order_after_current=True):
+        if not torch.cuda.is_available():
+            raise RuntimeError("DaSGD needs a CUDA device; there is no CPU implementation")
+        self.K, self.P, self.tau, self.d = K, P, tau, d
+        self.dtype = dtype
+        # True: before each step the main stream is made to wait (on the device) for torch's current
+        # stream, so gradients just produced by torch ops are complete.  Costs one event per call.
+        self.order_after_current = order_after_current
+        self.device = torch.device("cuda", device)
+        self.ld = ld if ld is not None else P
+        self.n_slots = n_slots if n_slots is not None else min_slots(tau, d)
+        dev = self.device
+        self.gdtype = torch.bfloat16 if dtype == DASGD_BF16_MASTER_F32 else torch.float32
+        self.w = torch.zeros((K, self.ld), dtype=torch.float32, device=dev)
+        self.m = torch.zeros((K, self.ld), dtype=torch.float32, device=dev) if momentum != 0.0 else None
+        self.w_lp = torch.zeros((K, self.ld), dtype=torch.bfloat16, device=dev) if dtype == DASGD_BF16_MASTER_F32 else None
+        self.snap = torch.empty((self.n_slots, K, self.ld), dtype=torch.float32, device=dev)
+        self.mean = torch.empty((self.n_slots, self.ld), dtype=torch.float32, device=dev)
+        self.g_stage = torch.empty((K, self.ld), dtype=self.gdtype, device=dev) if host_staging else None
+        try:
+            lo, hi = torch.cuda.Stream.priority_range()  # (least, greatest) priority
+        except Exception:
+            lo, hi = 0, -1
+        self.main = torch.cuda.Stream(device=dev, priority=lo)
+        self.side = torch.cuda.Stream(device=dev, priority=hi)
+        cfg = dasgd_config()
+        cfg.K, cfg.tau, cfg.d, cfg.dtype, cfg.merge_mode = K, tau, d, dtype, merge_mode
+        cfg.n_slots, cfg.flags, cfg.device, cfg.P, cfg.ld = self.n_slots, flags, dev.index or 0, P, self.ld
+        cfg.xi, cfg.momentum, cfg.weight_decay, cfg.sync_timeout_ms = xi, momentum, weight_decay, sync_timeout_ms
+        cfg.w = self.w.data_ptr()
+        cfg.m = self.m.data_ptr() if self.m is not None else None
+        cfg.w_lp = self.w_lp.data_ptr() if self.w_lp is not None else None
+        cfg.snap, cfg.mean = self.snap.data_ptr(), self.mean.data_ptr()
+        cfg.g_stage = self.g_stage.data_ptr() if self.g_stage is not None else None
+        cfg.main_stream, cfg.side_stream = self.main.cuda_stream, self.side.cuda_stream
+        self.cfg = cfg
+        torch.cuda.synchronize(dev)  # the zero fills above ran on torch's current stream
+        self.ctx = dasgd_init(cfg)
+
+    # -- state ---------------------------------------------------------------
+    def set_state(self, w, m=None):
+        """Copy initial weights ([P] shared start or [K, P]) and optionally momentum into the buffers."""
+        self.sync()  # work already queued on the library's streams must not race with the copies below
+        w = torch.as_tensor(w, dtype=torch.float32, device=self.device)
+        self.w[:, :self.P] = w if w.dim() == 2 else w.unsqueeze(0)
+        if m is not None and self.m is not None:
+            self.m[:, :self.P] = torch.as_tensor(m, dtype=torch.float32, device=self.device)
+        if self.w_lp is not None:
+            self.w_lp.copy_(self.w)  # round-to-nearest-even cast
+        torch.cuda.synchronize(self.device)
+
+    def _gptr(self, g: torch.Tensor) -> int:
+        if self.order_after_current:
+            self.main.wait_stream(torch.cuda.current_stream(self.device))
+        if g.dtype != self.gdtype or tuple(g.shape) != (self.K, self.ld) or not g.is_contiguous() or not g.is_cuda:
+            raise ValueError(f"gradients must be a contiguous CUDA {self.gdtype} tensor of shape {(self.K, self.ld)}")
+        return g.data_ptr()
+
+    # -- the path --------------------------------------------------------------
+    def local_step(self, g, lr):
+        dasgd_local_step(self.ctx, self._gptr(g), lr)
+
+    def snapshot(self):
+        dasgd_snapshot(self.ctx)
+
+    def average_async(self):
+        dasgd_average_async(self.ctx)
+
+    def merge(self):
+        dasgd_merge(self.ctx)
+
+    def sync(self):
+        dasgd_sync(self.ctx)
+
+    def step(self, g, lr):
+        dasgd_step(self.ctx, self._gptr(g), lr)
+
+    def step_host(self, g_host: torch.Tensor, lr, probe_host: torch.Tensor | None = None):
+        if g_host.is_cuda or g_host.dtype != self.gdtype or tuple(g_host.shape) != (self.K, self.ld):
+            raise ValueError("step_host wants a host tensor shaped like the gradients")
+        n = probe_host.numel() if probe_host is not None else 0
+        dasgd_step_host(self.ctx, g_host.data_ptr(), lr, probe_host.data_ptr() if n else None, n)
+
+    # -- introspection ---------------------------------------------------------
+    @property
+    def t(self):
+        return dasgd_get_step(self.ctx)[0]
+
+    @property
+    def n_pending(self):
+        return dasgd_get_step(self.ctx)[1]
+
+    def pending_mean(self, i=0) -> torch.Tensor:
+        """The mean vector of the i-th oldest pending snapshot (a view into ``self.mean``)."""
+        _, _, mean_ptr = dasgd_get_pending(self.ctx, i)
+        slot = (mean_ptr - self.mean.data_ptr()) // (self.ld * 4)
+        return self.mean[slot, :self.P]
+
+    def timing(self):
+        """(averages completed, ms spent averaging on the side stream, ms the main stream waited for them)."""
+        return dasgd_get_timing(self.ctx)
+
+    KERNELS = ("local_step", "snapshot", "mean", "merge", "stall")
+
+    def kernel_timing(self):
+        """{kind: (launches, total ms)} for the five kinds of timed work."""
+        return {name: dasgd_get_kernel_timing(self.ctx, i) for i, name in enumerate(self.KERNELS)}
+
+    def reset_timing(self):
+        dasgd_reset_timing(self.ctx)
+
+    @property
+    def launches(self):
+        return dasgd_get_launches(self.ctx)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            dasgd_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,672 @@
+// Host side of libdasgd: the C ABI declared in include/dasgd.h, the snapshot-slot state machine
+// and the two-stream scheduler that lets the worker-axis mean run beside the next local steps.
+#include "dasgd.h"
+#include "dasgd_kernels.cuh"
+
+#include <chrono>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <string>
+#include <thread>
+#include <vector>
+
+namespace {
+
+using dasgd::kThreads;
+using dasgd::Params;
+
+thread_local std::string g_init_error;
+
+enum SlotState { SLOT_FREE = 0, SLOT_SNAPPED = 1, SLOT_AVERAGING = 2 };
+
+struct Slot {
+  SlotState state = SLOT_FREE;
+  int64_t s = 0;                 // completed local steps when the snapshot was taken
+  cudaEvent_t e_snap = nullptr;  // main stream: snapshot written
+  cudaEvent_t e_avg = nullptr;   // side stream: mean written
+};
+
+// A pair of timing events around one piece of stream work, tagged with what it measures.
+enum SpanTag { TAG_STEP = 0, TAG_SNAPSHOT = 1, TAG_MEAN = 2, TAG_MERGE = 3, TAG_STALL = 4, TAG_COUNT = 5 };
+struct Span {
+  cudaEvent_t ev[2] = {nullptr, nullptr};
+  int tag = 0;
+  bool open = false;   // begin recorded, not yet harvested
+  bool ended = false;  // end recorded
+};
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace
+
+struct dasgd_ctx {
+  dasgd_config cfg;
+  cudaStream_t s0, s1;
+  int64_t t = 0;
+  int64_t launches = 0;
+  bool vec = false;  // rows are 16-byte aligned for every array: vector kernels usable
+  int epu = 4;       // elements per vector unit
+  std::vector<Slot> slots;
+  std::deque<int> pending;  // slot indices, oldest snapshot first
+  std::vector<Span> spans;
+  int64_t span_n[TAG_COUNT] = {0, 0, 0, 0, 0};
+  double span_ms[TAG_COUNT] = {0, 0, 0, 0, 0};
+  std::string err;
+};
+
+namespace {
+
+dasgd_status fail(dasgd_ctx *c, dasgd_status s, const std::string &msg) {
+  if (c) c->err = msg; else g_init_error = msg;
+  return s;
+}
+
+dasgd_status cuda_fail(dasgd_ctx *c, cudaError_t e, const char *what) {
+  return fail(c, DASGD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define CU(c, call)                                        \
+  do {                                                     \
+    cudaError_t e_ = (call);                               \
+    if (e_ != cudaSuccess) return cuda_fail(c, e_, #call); \
+  } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+float *snap_ptr(const dasgd_ctx *c, int slot) {
+  return static_cast<float *>(c->cfg.snap) + (size_t)slot * c->cfg.K * c->cfg.ld;
+}
+float *mean_ptr(const dasgd_ctx *c, int slot) {
+  return static_cast<float *>(c->cfg.mean) + (size_t)slot * c->cfg.ld;
+}
+
+Params base_params(const dasgd_ctx *c) {
+  Params p{};
+  p.w = static_cast<float *>(c->cfg.w);
+  p.m = static_cast<float *>(c->cfg.m);
+  p.w_lp = static_cast<__nv_bfloat16 *>(c->cfg.w_lp);
+  p.P = c->cfg.P;
+  p.ld = c->cfg.ld;
+  p.K = c->cfg.K;
+  p.mu = c->cfg.momentum;
+  p.lambda = c->cfg.weight_decay;
+  p.xi = c->cfg.xi;
+  p.omx = 1.0f - c->cfg.xi;
+  return p;
+}
+
+unsigned blocks_for(long long n, long long per_block) { return (unsigned)((n + per_block - 1) / per_block); }
+
+// -------------------------------------------------------------- timing bookkeeping
+
+void harvest(dasgd_ctx *c, bool block) {
+  for (Span &sp : c->spans) {
+    if (!sp.open || !sp.ended) continue;
+    if (block) {
+      if (cudaEventSynchronize(sp.ev[1]) != cudaSuccess) continue;
+    } else if (cudaEventQuery(sp.ev[1]) != cudaSuccess) {
+      cudaGetLastError();  // "not ready" is not an error here
+      continue;
+    }
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, sp.ev[0], sp.ev[1]) == cudaSuccess) {
+      c->span_n[sp.tag] += 1;
+      c->span_ms[sp.tag] += ms;
+    }
+    sp.open = sp.ended = false;
+  }
+}
+
+// Records the opening event of a span on `stream`; returns its index, or -1 when timing is off.
+int span_begin(dasgd_ctx *c, int tag, cudaStream_t stream) {
+  if (!(c->cfg.flags & DASGD_FLAG_TIMING)) return -1;
+  harvest(c, false);
+  int idx = -1;
+  for (size_t i = 0; i < c->spans.size(); ++i)
+    if (!c->spans[i].open) { idx = (int)i; break; }
+  if (idx < 0) {
+    Span sp;
+    if (cudaEventCreate(&sp.ev[0]) != cudaSuccess || cudaEventCreate(&sp.ev[1]) != cudaSuccess) return -1;
+    c->spans.push_back(sp);
+    idx = (int)c->spans.size() - 1;
+  }
+  Span &sp = c->spans[idx];
+  if (cudaEventRecord(sp.ev[0], stream) != cudaSuccess) return -1;
+  sp.tag = tag;
+  sp.open = true;
+  sp.ended = false;
+  return idx;
+}
+
+void span_end(dasgd_ctx *c, int idx, cudaStream_t stream) {
+  if (idx < 0) return;
+  if (cudaEventRecord(c->spans[idx].ev[1], stream) == cudaSuccess) c->spans[idx].ended = true;
+  else c->spans[idx].open = false;
+}
+
+// -------------------------------------------------------------- kernel launchers
+
+template <bool BF16, bool MOM, int MERGE, bool SNAP>
+dasgd_status launch_step_t(dasgd_ctx *c, const Params &p, bool vec) {
+  constexpr int EPU = BF16 ? 8 : 4;
+  constexpr int UNROLL = BF16 ? 2 : 4;
+  long long done = 0;
+  if (vec) {
+    const long long units = p.P / EPU;
+    if (units > 0) {
+      const long long tiles = (units + (long long)kThreads * UNROLL - 1) / ((long long)kThreads * UNROLL);
+      if (tiles * p.K > 0x7FFFFFFFLL) return fail(c, DASGD_ERR_UNSUPPORTED, "K*P too large for one launch");
+      dasgd::k_local_step_vec<BF16, MOM, MERGE, SNAP><<<(unsigned)(tiles * p.K), kThreads, 0, c->s0>>>(p);
+      c->launches++;
+    }
+    done = units * EPU;
+  }
+  if (done < p.P) {
+    dim3 grid(blocks_for(p.P - done, kThreads), (unsigned)p.K);
+    dasgd::k_local_step_scalar<BF16, MOM, MERGE, SNAP><<<grid, kThreads, 0, c->s0>>>(p, done);
+    c->launches++;
+  }
+  CU(c, cudaGetLastError());
+  return DASGD_OK;
+}
+
+template <bool BF16, bool MOM>
+dasgd_status launch_step_m(dasgd_ctx *c, const Params &p, bool vec, int merge, bool snap) {
+  switch (merge * 2 + (snap ? 1 : 0)) {
+    case 0: return launch_step_t<BF16, MOM, 0, false>(c, p, vec);
+    case 1: return launch_step_t<BF16, MOM, 0, true>(c, p, vec);
+    case 2: return launch_step_t<BF16, MOM, 1, false>(c, p, vec);
+    case 3: return launch_step_t<BF16, MOM, 1, true>(c, p, vec);
+    case 4: return launch_step_t<BF16, MOM, 2, false>(c, p, vec);
+    default: return launch_step_t<BF16, MOM, 2, true>(c, p, vec);
+  }
+}
+
+// merge: 0 none, 1 xi, 2 delta (fused into the step kernel); snap: also write p.snap_out
+dasgd_status launch_step(dasgd_ctx *c, const Params &p, bool vec, int merge, bool snap) {
+  const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32;
+  const bool mom = c->cfg.momentum != 0.0f;
+  const int sp = span_begin(c, TAG_STEP, c->s0);
+  dasgd_status st;
+  if (bf16) st = mom ? launch_step_m<true, true>(c, p, vec, merge, snap) : launch_step_m<true, false>(c, p, vec, merge, snap);
+  else st = mom ? launch_step_m<false, true>(c, p, vec, merge, snap) : launch_step_m<false, false>(c, p, vec, merge, snap);
+  span_end(c, sp, c->s0);
+  return st;
+}
+
+dasgd_status launch_snapshot(dasgd_ctx *c, const Params &p) {
+  const int sp = span_begin(c, TAG_SNAPSHOT, c->s0);
+  long long done = 0;
+  if (c->vec) {
+    const long long units = p.P / 4;
+    if (units > 0) {
+      const long long tiles = (units + (long long)kThreads * 4 - 1) / ((long long)kThreads * 4);
+      if (tiles * p.K > 0x7FFFFFFFLL) return fail(c, DASGD_ERR_UNSUPPORTED, "K*P too large for one launch");
+      dasgd::k_snapshot_vec<<<(unsigned)(tiles * p.K), kThreads, 0, c->s0>>>(p);
+      c->launches++;
+    }
+    done = units * 4;
+  }
+  if (done < p.P) {
+    dim3 grid(blocks_for(p.P - done, kThreads), (unsigned)p.K);
+    dasgd::k_snapshot_scalar<<<grid, kThreads, 0, c->s0>>>(p, done);
+    c->launches++;
+  }
+  span_end(c, sp, c->s0);
+  CU(c, cudaGetLastError());
+  return DASGD_OK;
+}
+
+dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
+  const int sp = span_begin(c, TAG_MEAN, c->s1);
+  long long done = 0;
+  if (c->vec) {
+    const long long units = p.P / 4;
+    if (units > 0) {
+      dasgd::k_reduce_vec<<<blocks_for(units, kThreads), kThreads, 0, c->s1>>>(p);
+      c->launches++;
+    }
+    done = units * 4;
+  }
+  if (done < p.P) {
+    dasgd::k_reduce_scalar<<<blocks_for(p.P - done, kThreads), kThreads, 0, c->s1>>>(p, done);
+    c->launches++;
+  }
+  span_end(c, sp, c->s1);
+  CU(c, cudaGetLastError());
+  return DASGD_OK;
+}
+
+template <bool BF16, int MODE, bool SNAP>
+dasgd_status launch_merge_t(dasgd_ctx *c, const Params &p) {
+  constexpr int EPU = BF16 ? 8 : 4;
+  const int sp = span_begin(c, TAG_MERGE, c->s0);
+  long long done = 0;
+  if (c->vec) {
+    const long long units = p.P / EPU;
+    if (units > 0) {
+      dasgd::k_merge_vec<BF16, MODE, SNAP><<<blocks_for(units, kThreads), kThreads, 0, c->s0>>>(p);
+      c->launches++;
+    }
+    done = units * EPU;
+  }
+  if (done < p.P) {
+    dasgd::k_merge_scalar<BF16, MODE, SNAP><<<blocks_for(p.P - done, kThreads), kThreads, 0, c->s0>>>(p, done);
+    c->launches++;
+  }
+  span_end(c, sp, c->s0);
+  CU(c, cudaGetLastError());
+  return DASGD_OK;
+}
+
+dasgd_status launch_merge(dasgd_ctx *c, const Params &p, bool snap) {
+  const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32;
+  const bool delta = c->cfg.merge_mode == DASGD_MERGE_DELTA;
+  if (bf16) {
+    if (delta) return snap ? launch_merge_t<true, 2, true>(c, p) : launch_merge_t<true, 2, false>(c, p);
+    return snap ? launch_merge_t<true, 1, true>(c, p) : launch_merge_t<true, 1, false>(c, p);
+  }
+  if (delta) return snap ? launch_merge_t<false, 2, true>(c, p) : launch_merge_t<false, 2, false>(c, p);
+  return snap ? launch_merge_t<false, 1, true>(c, p) : launch_merge_t<false, 1, false>(c, p);
+}
+
+// -------------------------------------------------------------- slot operations
+
+int find_free_slot(const dasgd_ctx *c) {
+  for (size_t i = 0; i < c->slots.size(); ++i)
+    if (c->slots[i].state == SLOT_FREE) return (int)i;
+  return -1;
+}
+
+// book-keeping after the main stream has been given the work that writes snap[slot]
+dasgd_status mark_snapped(dasgd_ctx *c, int slot) {
+  Slot &sl = c->slots[slot];
+  CU(c, cudaEventRecord(sl.e_snap, c->s0));
+  sl.state = SLOT_SNAPPED;
+  sl.s = c->t;
+  c->pending.push_back(slot);
+  return DASGD_OK;
+}
+
+// make the main stream wait for the oldest pending average; returns its slot
+dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
+  if (c->pending.empty()) return fail(c, DASGD_ERR_BAD_STATE, "merge: no snapshot is pending");
+  const int slot = c->pending.front();
+  Slot &sl = c->slots[slot];
+  if (sl.state != SLOT_AVERAGING)
+    return fail(c, DASGD_ERR_BAD_STATE, "merge: the oldest snapshot has not been given to dasgd_average_async");
+  const int sp = span_begin(c, TAG_STALL, c->s0);
+  CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg, 0));
+  span_end(c, sp, c->s0);
+  *slot_out = slot;
+  return DASGD_OK;
+}
+
+void release_oldest(dasgd_ctx *c) {
+  const int slot = c->pending.front();
+  c->pending.pop_front();
+  c->slots[slot].state = SLOT_FREE;
+}
+
+bool merge_due(const dasgd_ctx *c, int64_t u) {
+  const int64_t tau = c->cfg.tau, d = c->cfg.d;
+  return d > 0 && u - d >= tau && (u - d) % tau == 0;
+}
+
+bool grads_vec_ok(const dasgd_ctx *c, const void *g) { return c->vec && aligned16(g); }
+
+dasgd_status do_average(dasgd_ctx *c) {
+  int slot = -1;
+  for (int s : c->pending)
+    if (c->slots[s].state == SLOT_SNAPPED) { slot = s; break; }
+  if (slot < 0) return fail(c, DASGD_ERR_BAD_STATE, "average: no snapshot is waiting for its mean");
+  Slot &sl = c->slots[slot];
+  CU(c, cudaStreamWaitEvent(c->s1, sl.e_snap, 0));
+  Params p = base_params(c);
+  p.snap_in = snap_ptr(c, slot);
+  p.mean_out = mean_ptr(c, slot);
+  dasgd_status st = launch_reduce(c, p);
+  if (st != DASGD_OK) return st;
+  CU(c, cudaEventRecord(sl.e_avg, c->s1));
+  sl.state = SLOT_AVERAGING;
+  return DASGD_OK;
+}
+
+}  // namespace
+
+// ================================================================== C ABI
+
+extern "C" {
+
+const char *dasgd_version(void) { return "0.1"; }
+
+const char *dasgd_strerror(dasgd_status s) {
+  switch (s) {
+    case DASGD_OK: return "ok";
+    case DASGD_ERR_INVALID_ARG: return "invalid argument";
+    case DASGD_ERR_BAD_STATE: return "call out of order";
+    case DASGD_ERR_NO_SLOT: return "no free snapshot slot";
+    case DASGD_ERR_CUDA: return "CUDA error";
+    case DASGD_ERR_TIMEOUT: return "timed out";
+    case DASGD_ERR_UNSUPPORTED: return "unsupported";
+  }
+  return "unknown status";
+}
+
+const char *dasgd_last_error(const dasgd_ctx *ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
+  if (!out) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: out is NULL");
+  *out = nullptr;
+  if (!cfg) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: cfg is NULL");
+  dasgd_config c = *cfg;
+  if (c.ld == 0) c.ld = c.P;
+  if (c.K < 1 || c.K > 65535) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: K must be in [1, 65535]");
+  if (c.P < 1) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: P must be >= 1");
+  if (c.ld < c.P) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: ld must be >= P");
+  if (c.tau < 1) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: tau must be >= 1");
+  if (c.d < 0) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: d must be >= 0");
+  if (!(c.xi >= 0.0f && c.xi <= 1.0f)) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: xi must be in [0, 1]");
+  if (!(c.momentum >= 0.0f) || !(c.weight_decay >= 0.0f))
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: momentum and weight_decay must be >= 0");
+  if (c.dtype != DASGD_F32 && c.dtype != DASGD_BF16_MASTER_F32)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: unknown dtype");
+  if (c.merge_mode != DASGD_MERGE_XI && c.merge_mode != DASGD_MERGE_DELTA)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: unknown merge_mode");
+  const int need = c.d == 0 ? 1 : (c.d + c.tau - 1) / c.tau;
+  if (c.n_slots < need)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: n_slots must be >= max(1, ceil(d/tau))");
+  if (!c.w || !c.snap || !c.mean) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: w, snap and mean must not be NULL");
+  if (c.momentum != 0.0f && !c.m) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: momentum != 0 needs m");
+  if (c.dtype == DASGD_BF16_MASTER_F32 && !c.w_lp)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: bf16 mode needs w_lp");
+  const void *ptrs[] = {c.w, c.m, c.w_lp, c.snap, c.mean, c.g_stage};
+  for (const void *p : ptrs)
+    if (p && !aligned16(p)) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: device buffers must be 16-byte aligned");
+  if (c.main_stream == c.side_stream)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: main_stream and side_stream must differ");
+  if (c.sync_timeout_ms == 0) c.sync_timeout_ms = 60000;
+
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess) return cuda_fail(nullptr, e, "init: cudaGetDeviceCount");
+  if (c.device < 0 || c.device >= ndev) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: no such CUDA device");
+
+  dasgd_ctx *ctx = new (std::nothrow) dasgd_ctx();
+  if (!ctx) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: out of host memory");
+  ctx->cfg = c;
+  ctx->s0 = static_cast<cudaStream_t>(c.main_stream);
+  ctx->s1 = static_cast<cudaStream_t>(c.side_stream);
+  ctx->epu = c.dtype == DASGD_BF16_MASTER_F32 ? 8 : 4;
+  ctx->vec = (c.ld % ctx->epu) == 0;
+  DeviceGuard guard(c.device);
+  ctx->slots.resize(c.n_slots);
+  for (Slot &sl : ctx->slots) {
+    if ((e = cudaEventCreateWithFlags(&sl.e_snap, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&sl.e_avg, cudaEventDisableTiming)) != cudaSuccess) {
+      dasgd_status st = cuda_fail(nullptr, e, "init: cudaEventCreate");
+      for (Slot &z : ctx->slots) {
+        if (z.e_snap) cudaEventDestroy(z.e_snap);
+        if (z.e_avg) cudaEventDestroy(z.e_avg);
+      }
+      delete ctx;
+      return st;
+    }
+  }
+  *out = ctx;
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  cudaStreamSynchronize(ctx->s0);
+  cudaStreamSynchronize(ctx->s1);
+  for (Slot &sl : ctx->slots) {
+    if (sl.e_snap) cudaEventDestroy(sl.e_snap);
+    if (sl.e_avg) cudaEventDestroy(sl.e_avg);
+  }
+  for (Span &sp : ctx->spans)
+    for (int j = 0; j < 2; ++j)
+      if (sp.ev[j]) cudaEventDestroy(sp.ev[j]);
+  delete ctx;
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_local_step(dasgd_ctx *ctx, const void *grads, float lr) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!grads) return fail(ctx, DASGD_ERR_INVALID_ARG, "local_step: grads is NULL");
+  DeviceGuard guard(ctx->cfg.device);
+  Params p = base_params(ctx);
+  p.g = grads;
+  p.lr = lr;
+  dasgd_status st = launch_step(ctx, p, grads_vec_ok(ctx, grads), 0, false);
+  if (st == DASGD_OK) ctx->t += 1;
+  return st;
+}
+
+dasgd_status dasgd_snapshot(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  const int slot = find_free_slot(ctx);
+  if (slot < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "snapshot: every slot holds a pending average");
+  Params p = base_params(ctx);
+  p.snap_out = snap_ptr(ctx, slot);
+  dasgd_status st = launch_snapshot(ctx, p);
+  if (st != DASGD_OK) return st;
+  return mark_snapped(ctx, slot);
+}
+
+dasgd_status dasgd_average_async(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  return do_average(ctx);
+}
+
+dasgd_status dasgd_merge(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  int slot = -1;
+  dasgd_status st = wait_oldest_average(ctx, &slot);
+  if (st != DASGD_OK) return st;
+  Params p = base_params(ctx);
+  p.mean = mean_ptr(ctx, slot);
+  p.snap_in = snap_ptr(ctx, slot);
+  st = launch_merge(ctx, p, false);
+  if (st != DASGD_OK) return st;
+  release_oldest(ctx);
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!grads) return fail(ctx, DASGD_ERR_INVALID_ARG, "step: grads is NULL");
+  DeviceGuard guard(ctx->cfg.device);
+  const dasgd_config &cfg = ctx->cfg;
+  const int64_t u = ctx->t + 1;
+  const bool m_due = merge_due(ctx, u);
+  const bool s_due = (u % cfg.tau) == 0;
+  const bool fuse_merge = m_due && (cfg.flags & DASGD_FLAG_FUSE_MERGE) && cfg.d >= 2;
+  const bool fuse_snap = s_due && (cfg.flags & DASGD_FLAG_FUSE_SNAPSHOT);
+  const int mode = cfg.merge_mode == DASGD_MERGE_DELTA ? 2 : 1;
+  dasgd_status st;
+
+  // The snapshot of this iteration may reuse the slot whose mean is merged in this same iteration:
+  // each thread reads the old snapshot/mean elements before it overwrites them.
+  int merge_slot = -1, snap_slot = -1;
+  Params p = base_params(ctx);
+  p.g = grads;
+  p.lr = lr;
+
+  // ---- local step (optionally with the merge and/or the snapshot store folded in)
+  if (fuse_merge) {
+    st = wait_oldest_average(ctx, &merge_slot);
+    if (st != DASGD_OK) return st;
+    p.mean = mean_ptr(ctx, merge_slot);
+    p.snap_in = snap_ptr(ctx, merge_slot);
+  }
+  const bool step_writes_snap = fuse_snap && (!m_due || fuse_merge);
+  if (step_writes_snap) {
+    snap_slot = fuse_merge ? merge_slot : find_free_slot(ctx);
+    if (snap_slot < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot slot");
+    p.snap_out = snap_ptr(ctx, snap_slot);
+  }
+  st = launch_step(ctx, p, grads_vec_ok(ctx, grads), fuse_merge ? mode : 0, step_writes_snap);
+  if (st != DASGD_OK) return st;
+  ctx->t = u;
+  if (fuse_merge) release_oldest(ctx);
+
+  // ---- separate merge kernel (d == 1, or fusion off), optionally storing the snapshot
+  if (m_due && !fuse_merge) {
+    st = wait_oldest_average(ctx, &merge_slot);
+    if (st != DASGD_OK) return st;
+    Params q = base_params(ctx);
+    q.mean = mean_ptr(ctx, merge_slot);
+    q.snap_in = snap_ptr(ctx, merge_slot);
+    if (fuse_snap) {
+      snap_slot = merge_slot;
+      q.snap_out = snap_ptr(ctx, snap_slot);
+    }
+    st = launch_merge(ctx, q, fuse_snap);
+    if (st != DASGD_OK) return st;
+    release_oldest(ctx);
+  }
+
+  // ---- snapshot and its mean
+  if (s_due) {
+    if (snap_slot >= 0) {
+      st = mark_snapped(ctx, snap_slot);
+    } else {
+      const int slot = find_free_slot(ctx);
+      if (slot < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot slot");
+      Params q = base_params(ctx);
+      q.snap_out = snap_ptr(ctx, slot);
+      st = launch_snapshot(ctx, q);
+      if (st == DASGD_OK) st = mark_snapped(ctx, slot);
+    }
+    if (st != DASGD_OK) return st;
+    st = do_average(ctx);
+    if (st != DASGD_OK) return st;
+    if (cfg.d == 0) {  // Local SGD: the mean is applied in the same iteration
+      int slot = -1;
+      st = wait_oldest_average(ctx, &slot);
+      if (st != DASGD_OK) return st;
+      Params q = base_params(ctx);
+      q.mean = mean_ptr(ctx, slot);
+      q.snap_in = snap_ptr(ctx, slot);
+      st = launch_merge(ctx, q, false);
+      if (st != DASGD_OK) return st;
+      release_oldest(ctx);
+    }
+  }
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_step_host(dasgd_ctx *ctx, const void *grads_host, float lr, float *probe_host,
+                             int64_t probe_elems) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!grads_host) return fail(ctx, DASGD_ERR_INVALID_ARG, "step_host: grads_host is NULL");
+  if (!ctx->cfg.g_stage) return fail(ctx, DASGD_ERR_BAD_STATE, "step_host: cfg.g_stage was NULL");
+  if (probe_host && (probe_elems < 0 || probe_elems > ctx->cfg.P))
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "step_host: probe_elems must be in [0, P]");
+  DeviceGuard guard(ctx->cfg.device);
+  const size_t esz = ctx->cfg.dtype == DASGD_BF16_MASTER_F32 ? 2 : 4;
+  const size_t bytes = (size_t)ctx->cfg.K * ctx->cfg.ld * esz;
+  CU(ctx, cudaMemcpyAsync(ctx->cfg.g_stage, grads_host, bytes, cudaMemcpyHostToDevice, ctx->s0));
+  dasgd_status st = dasgd_step(ctx, ctx->cfg.g_stage, lr);
+  if (st != DASGD_OK) return st;
+  if (probe_host && probe_elems > 0)
+    CU(ctx, cudaMemcpyAsync(probe_host, ctx->cfg.w, (size_t)probe_elems * sizeof(float), cudaMemcpyDeviceToHost,
+                            ctx->s0));
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_sync(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(ctx->cfg.sync_timeout_ms);
+  cudaStream_t streams[2] = {ctx->s0, ctx->s1};
+  for (cudaStream_t s : streams) {
+    for (;;) {
+      cudaError_t e = cudaStreamQuery(s);
+      if (e == cudaSuccess) break;
+      if (e != cudaErrorNotReady) return cuda_fail(ctx, e, "sync: cudaStreamQuery");
+      if (std::chrono::steady_clock::now() > deadline)
+        return fail(ctx, DASGD_ERR_TIMEOUT, "sync: streams still busy after sync_timeout_ms");
+      std::this_thread::sleep_for(std::chrono::microseconds(20));
+    }
+  }
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_step(const dasgd_ctx *ctx, int64_t *t, int32_t *pending) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (t) *t = ctx->t;
+  if (pending) *pending = (int32_t)ctx->pending.size();
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_pending(const dasgd_ctx *ctx, int32_t i, int64_t *s, void **snap_device, void **mean_device) {
+  if (!ctx || i < 0 || i >= (int32_t)ctx->pending.size()) return DASGD_ERR_INVALID_ARG;
+  const int slot = ctx->pending[i];
+  if (s) *s = ctx->slots[slot].s;
+  if (snap_device) *snap_device = snap_ptr(ctx, slot);
+  if (mean_device) *mean_device = mean_ptr(ctx, slot);
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_timing(dasgd_ctx *ctx, int64_t *n_avg, double *ms_avg, double *ms_stall) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!(ctx->cfg.flags & DASGD_FLAG_TIMING)) return fail(ctx, DASGD_ERR_BAD_STATE, "get_timing: DASGD_FLAG_TIMING not set");
+  dasgd_status st = dasgd_sync(ctx);
+  if (st != DASGD_OK) return st;
+  DeviceGuard guard(ctx->cfg.device);
+  harvest(ctx, true);
+  if (n_avg) *n_avg = ctx->span_n[TAG_MEAN];
+  if (ms_avg) *ms_avg = ctx->span_ms[TAG_MEAN];
+  if (ms_stall) *ms_stall = ctx->span_ms[TAG_STALL];
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_kernel_timing(dasgd_ctx *ctx, int32_t which, int64_t *n, double *ms) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (which < 0 || which >= TAG_COUNT) return fail(ctx, DASGD_ERR_INVALID_ARG, "get_kernel_timing: which must be in [0, 4]");
+  if (!(ctx->cfg.flags & DASGD_FLAG_TIMING))
+    return fail(ctx, DASGD_ERR_BAD_STATE, "get_kernel_timing: DASGD_FLAG_TIMING not set");
+  dasgd_status st = dasgd_sync(ctx);
+  if (st != DASGD_OK) return st;
+  DeviceGuard guard(ctx->cfg.device);
+  harvest(ctx, true);
+  if (n) *n = ctx->span_n[which];
+  if (ms) *ms = ctx->span_ms[which];
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_reset_timing(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  dasgd_status st = dasgd_sync(ctx);
+  if (st != DASGD_OK) return st;
+  DeviceGuard guard(ctx->cfg.device);
+  harvest(ctx, true);
+  for (int i = 0; i < TAG_COUNT; ++i) { ctx->span_n[i] = 0; ctx->span_ms[i] = 0.0; }
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches) {
+  if (!ctx || !launches) return DASGD_ERR_INVALID_ARG;
+  *launches = ctx->launches;
+  return DASGD_OK;
+}
+
+}  // extern "C"

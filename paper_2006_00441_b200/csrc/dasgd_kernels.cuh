@@ -1,0 +1,330 @@
+// Device code of libdasgd: the four element-wise / worker-axis kernels of the DaSGD hot path.
+//
+// Every operation is independent across the parameter index p and moves each byte once, so the
+// kernels are HBM-bandwidth bound: the work is laid out for coalesced 128-bit accesses with many
+// independent loads in flight per thread, streaming cache hints (nothing is reused inside a
+// kernel), and small CTAs so that a higher-priority side-stream kernel can take SM slots as they
+// retire.  Tensor cores have no role here (about 0.2 flop per byte).
+//
+// Arithmetic is float32 with explicit fused multiply-adds, the same expressions in every
+// variant, so that fused and unfused schedules give bit-identical results:
+//     g' = fma(lambda, w, g);  m = fma(mu, m, g');  w = fma(-lr, m, w)        (local step)
+//     w  = fma(xi, w, (1-xi)*mean)                                            (xi merge)
+//     w  = w + (mean - snap)                                                  (delta merge)
+//     mean = (pairwise sum over k) / K                                        (worker-axis mean)
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dasgd {
+
+constexpr int kThreads = 256;
+
+struct Params {
+  float *w;             // [K][ld]
+  float *m;             // [K][ld] or nullptr
+  const void *g;        // [K][ld] float or bf16
+  __nv_bfloat16 *w_lp;  // [K][ld] or nullptr
+  float *snap_out;      // [K][ld] snapshot slot to write, or nullptr
+  const float *snap_in; // [K][ld] snapshot slot to read (delta merge), or nullptr
+  const float *mean;    // [ld] mean slot to read, or nullptr
+  float *mean_out;      // [ld] mean slot to write (reduce)
+  long long P, ld;
+  int K;
+  float lr, mu, lambda, xi, omx;
+};
+
+// ---------------------------------------------------------------- memory helpers
+
+__device__ __forceinline__ float4 ld_stream(const float4 *p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4 *p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4 *p, uint4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
+
+// two float32 -> packed bf16x2, round to nearest even (lo in the low half)
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// ---------------------------------------------------------------- scalar arithmetic
+
+template <bool MOM>
+__device__ __forceinline__ void step_elem(float &w, float &m, float g, const Params &p) {
+  const float gp = fmaf(p.lambda, w, g);
+  if (MOM) {
+    m = fmaf(p.mu, m, gp);
+    w = fmaf(-p.lr, m, w);
+  } else {
+    w = fmaf(-p.lr, gp, w);
+  }
+}
+
+__device__ __forceinline__ float blend_xi(float w, float mean, const Params &p) {
+  return fmaf(p.xi, w, __fmul_rn(p.omx, mean));
+}
+
+__device__ __forceinline__ float blend_delta(float w, float mean, float snap) {
+  return __fadd_rn(w, __fsub_rn(mean, snap));
+}
+
+#define DASGD_F4_APPLY(dst, expr_x, expr_y, expr_z, expr_w) \
+  dst.x = expr_x; dst.y = expr_y; dst.z = expr_z; dst.w = expr_w;
+
+// ---------------------------------------------------------------- local step (vector path)
+//
+// One CTA = one worker k and one tile of kThreads*UNROLL units; a unit is 4 (float32 gradients) or
+// 8 (bfloat16 gradients) consecutive parameters.  blockIdx.x enumerates (tile, k) with k fastest so
+// that CTAs sharing a mean tile (fused merge) are neighbours in launch order.
+// MERGE: 0 none, 1 xi-blend, 2 delta.  SNAP: also store the final w into snap_out.
+
+template <bool BF16, bool MOM, int MERGE, bool SNAP>
+__global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
+  constexpr int EPU = BF16 ? 8 : 4;   // elements per unit
+  constexpr int F4 = EPU / 4;          // float4 per unit
+  constexpr int UNROLL = BF16 ? 2 : 4; // units per thread
+  const int k = blockIdx.x % p.K;
+  const long long tile = blockIdx.x / p.K;
+  const long long units = p.P / EPU;
+  const long long row = (long long)k * p.ld;
+  const long long u0 = tile * (long long)(kThreads * UNROLL) + threadIdx.x;
+
+  float4 w4[UNROLL][F4], m4[UNROLL][F4], g4[UNROLL][F4], a4[UNROLL][F4], s4[UNROLL][F4];
+  bool ok[UNROLL];
+
+#pragma unroll
+  for (int j = 0; j < UNROLL; ++j) {
+    const long long u = u0 + (long long)j * kThreads;
+    ok[j] = u < units;
+    if (ok[j]) {
+      const long long e = u * EPU;  // element offset inside the row
+      if (BF16) {
+        const uint4 gb = ld_stream(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.g) + row + e));
+        g4[j][0] = make_float4(bf16_bits_to_f32(gb.x & 0xFFFFu), bf16_bits_to_f32(gb.x >> 16),
+                               bf16_bits_to_f32(gb.y & 0xFFFFu), bf16_bits_to_f32(gb.y >> 16));
+        g4[j][F4 - 1] = make_float4(bf16_bits_to_f32(gb.z & 0xFFFFu), bf16_bits_to_f32(gb.z >> 16),
+                                    bf16_bits_to_f32(gb.w & 0xFFFFu), bf16_bits_to_f32(gb.w >> 16));
+      } else {
+        g4[j][0] = ld_stream(reinterpret_cast<const float4 *>(static_cast<const float *>(p.g) + row + e));
+      }
+#pragma unroll
+      for (int f = 0; f < F4; ++f) {
+        w4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.w + row + e) + f);
+        if (MOM) m4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.m + row + e) + f);
+        if (MERGE != 0) a4[j][f] = __ldg(reinterpret_cast<const float4 *>(p.mean + e) + f);
+        if (MERGE == 2) s4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.snap_in + row + e) + f);
+      }
+    }
+  }
+
+#pragma unroll
+  for (int j = 0; j < UNROLL; ++j) {
+    if (!ok[j]) continue;
+    const long long e = (u0 + (long long)j * kThreads) * EPU;
+#pragma unroll
+    for (int f = 0; f < F4; ++f) {
+      float4 w = w4[j][f];
+      float4 m = MOM ? m4[j][f] : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 g = g4[j][f];
+      step_elem<MOM>(w.x, m.x, g.x, p);
+      step_elem<MOM>(w.y, m.y, g.y, p);
+      step_elem<MOM>(w.z, m.z, g.z, p);
+      step_elem<MOM>(w.w, m.w, g.w, p);
+      if (MERGE == 1) {
+        const float4 a = a4[j][f];
+        DASGD_F4_APPLY(w, blend_xi(w.x, a.x, p), blend_xi(w.y, a.y, p), blend_xi(w.z, a.z, p), blend_xi(w.w, a.w, p))
+      } else if (MERGE == 2) {
+        const float4 a = a4[j][f], s = s4[j][f];
+        DASGD_F4_APPLY(w, blend_delta(w.x, a.x, s.x), blend_delta(w.y, a.y, s.y), blend_delta(w.z, a.z, s.z),
+                       blend_delta(w.w, a.w, s.w))
+      }
+      st_stream(reinterpret_cast<float4 *>(p.w + row + e) + f, w);
+      if (MOM) st_stream(reinterpret_cast<float4 *>(p.m + row + e) + f, m);
+      if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + row + e) + f, w);
+      w4[j][f] = w;
+    }
+    if (BF16) {
+      uint4 o;
+      o.x = pack_bf16x2(w4[j][0].x, w4[j][0].y);
+      o.y = pack_bf16x2(w4[j][0].z, w4[j][0].w);
+      o.z = pack_bf16x2(w4[j][F4 - 1].x, w4[j][F4 - 1].y);
+      o.w = pack_bf16x2(w4[j][F4 - 1].z, w4[j][F4 - 1].w);
+      st_stream(reinterpret_cast<uint4 *>(p.w_lp + row + e), o);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- local step (scalar path)
+// Columns [p0, P) of every row, one thread per (k, p).  Used for the ragged end of a row and for
+// arrays whose rows are not 16-byte aligned.
+
+template <bool BF16, bool MOM, int MERGE, bool SNAP>
+__global__ void __launch_bounds__(kThreads) k_local_step_scalar(const Params p, long long p0) {
+  const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
+  const int k = blockIdx.y;
+  if (col >= p.P) return;
+  const long long i = (long long)k * p.ld + col;
+  float w = p.w[i], m = MOM ? p.m[i] : 0.0f;
+  const float g = BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(p.g)[i])
+                       : static_cast<const float *>(p.g)[i];
+  step_elem<MOM>(w, m, g, p);
+  if (MERGE == 1) w = blend_xi(w, p.mean[col], p);
+  if (MERGE == 2) w = blend_delta(w, p.mean[col], p.snap_in[i]);
+  p.w[i] = w;
+  if (MOM) p.m[i] = m;
+  if (SNAP) p.snap_out[i] = w;
+  if (BF16) p.w_lp[i] = __float2bfloat16_rn(w);
+}
+
+// ---------------------------------------------------------------- snapshot copy
+
+__global__ void __launch_bounds__(kThreads) k_snapshot_vec(const Params p) {
+  constexpr int UNROLL = 4;
+  const int k = blockIdx.x % p.K;
+  const long long tile = blockIdx.x / p.K;
+  const long long units = p.P / 4;
+  const long long row = (long long)k * p.ld;
+  const long long u0 = tile * (long long)(kThreads * UNROLL) + threadIdx.x;
+  float4 v[UNROLL];
+#pragma unroll
+  for (int j = 0; j < UNROLL; ++j) {
+    const long long u = u0 + (long long)j * kThreads;
+    if (u < units) v[j] = ld_stream(reinterpret_cast<const float4 *>(p.w + row) + u);
+  }
+#pragma unroll
+  for (int j = 0; j < UNROLL; ++j) {
+    const long long u = u0 + (long long)j * kThreads;
+    if (u < units) st_stream(reinterpret_cast<float4 *>(p.snap_out + row) + u, v[j]);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) k_snapshot_scalar(const Params p, long long p0) {
+  const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (col >= p.P) return;
+  const long long i = (long long)blockIdx.y * p.ld + col;
+  p.snap_out[i] = p.w[i];
+}
+
+// ---------------------------------------------------------------- worker-axis mean
+// One thread owns 4 consecutive parameters and walks the K rows, eight independent 16-byte loads
+// at a time.  Summation: four interleaved partial sums (k mod 4) combined pairwise; then one
+// correctly rounded division by K.
+
+__device__ __forceinline__ void add4(float4 &a, const float4 &b) {
+  a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y); a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
+}
+
+__global__ void __launch_bounds__(kThreads) k_reduce_vec(const Params p) {
+  const long long u = (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (u >= p.P / 4) return;
+  const float4 *base = reinterpret_cast<const float4 *>(p.snap_in) + u;
+  const long long ld4 = p.ld / 4;
+  float4 acc[4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a) acc[a] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k0 = 0; k0 < p.K; k0 += 8) {
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (k0 + j < p.K) v[j] = ld_stream(base + (long long)(k0 + j) * ld4);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (k0 + j < p.K) add4(acc[j & 3], v[j]);
+  }
+  add4(acc[0], acc[1]);
+  add4(acc[2], acc[3]);
+  add4(acc[0], acc[2]);
+  const float kf = (float)p.K;
+  float4 r;
+  r.x = __fdiv_rn(acc[0].x, kf); r.y = __fdiv_rn(acc[0].y, kf);
+  r.z = __fdiv_rn(acc[0].z, kf); r.w = __fdiv_rn(acc[0].w, kf);
+  reinterpret_cast<float4 *>(p.mean_out)[u] = r;  // re-read by the merge: leave it cacheable
+}
+
+__global__ void __launch_bounds__(kThreads) k_reduce_scalar(const Params p, long long p0) {
+  const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (col >= p.P) return;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int k = 0; k < p.K; ++k) acc[k & 3] = __fadd_rn(acc[k & 3], p.snap_in[(long long)k * p.ld + col]);
+  const float s = __fadd_rn(__fadd_rn(acc[0], acc[1]), __fadd_rn(acc[2], acc[3]));
+  p.mean_out[col] = __fdiv_rn(s, (float)p.K);
+}
+
+// ---------------------------------------------------------------- delayed merge
+// One thread owns one unit of the parameter axis, keeps the mean in registers and walks the K
+// rows four at a time: the mean is read from HBM once, not K times.
+
+template <bool BF16, int MODE /*1 xi, 2 delta*/, bool SNAP>
+__global__ void __launch_bounds__(kThreads) k_merge_vec(const Params p) {
+  constexpr int EPU = BF16 ? 8 : 4;
+  constexpr int F4 = EPU / 4;
+  constexpr int KB = BF16 ? 2 : 4;  // rows in flight
+  const long long u = (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (u >= p.P / EPU) return;
+  const long long e = u * EPU;
+  float4 a[F4];
+#pragma unroll
+  for (int f = 0; f < F4; ++f) a[f] = __ldg(reinterpret_cast<const float4 *>(p.mean + e) + f);
+  for (int k0 = 0; k0 < p.K; k0 += KB) {
+    float4 w[KB][F4], s[KB][F4];
+#pragma unroll
+    for (int j = 0; j < KB; ++j) {
+      if (k0 + j >= p.K) continue;
+      const long long off = (long long)(k0 + j) * p.ld + e;
+#pragma unroll
+      for (int f = 0; f < F4; ++f) {
+        w[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.w + off) + f);
+        if (MODE == 2) s[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.snap_in + off) + f);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < KB; ++j) {
+      if (k0 + j >= p.K) continue;
+      const long long off = (long long)(k0 + j) * p.ld + e;
+#pragma unroll
+      for (int f = 0; f < F4; ++f) {
+        float4 x = w[j][f];
+        if (MODE == 1) {
+          DASGD_F4_APPLY(x, blend_xi(x.x, a[f].x, p), blend_xi(x.y, a[f].y, p), blend_xi(x.z, a[f].z, p),
+                         blend_xi(x.w, a[f].w, p))
+        } else {
+          const float4 t = s[j][f];
+          DASGD_F4_APPLY(x, blend_delta(x.x, a[f].x, t.x), blend_delta(x.y, a[f].y, t.y),
+                         blend_delta(x.z, a[f].z, t.z), blend_delta(x.w, a[f].w, t.w))
+        }
+        st_stream(reinterpret_cast<float4 *>(p.w + off) + f, x);
+        if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + off) + f, x);
+        w[j][f] = x;
+      }
+      if (BF16) {
+        uint4 o;
+        o.x = pack_bf16x2(w[j][0].x, w[j][0].y);
+        o.y = pack_bf16x2(w[j][0].z, w[j][0].w);
+        o.z = pack_bf16x2(w[j][F4 - 1].x, w[j][F4 - 1].y);
+        o.w = pack_bf16x2(w[j][F4 - 1].z, w[j][F4 - 1].w);
+        st_stream(reinterpret_cast<uint4 *>(p.w_lp + off), o);
+      }
+    }
+  }
+}
+
+template <bool BF16, int MODE, bool SNAP>
+__global__ void __launch_bounds__(kThreads) k_merge_scalar(const Params p, long long p0) {
+  const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (col >= p.P) return;
+  const float a = p.mean[col];
+  for (int k = 0; k < p.K; ++k) {
+    const long long i = (long long)k * p.ld + col;
+    float w = p.w[i];
+    w = (MODE == 1) ? blend_xi(w, a, p) : blend_delta(w, a, p.snap_in[i]);
+    p.w[i] = w;
+    if (SNAP) p.snap_out[i] = w;
+    if (BF16) p.w_lp[i] = __float2bfloat16_rn(w);
+  }
+}
+
+}  // namespace dasgd

@@ -1,0 +1,67 @@
+"""The C-ABI library loads without a GPU, exports every declared symbol, and validates arguments."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2006_00441_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "dasgd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dasgd_[a-z_]+)\s*\(", text)))
+
+
+def test_header_and_library_agree_on_exports():
+    names = declared_symbols()
+    assert set(names) == set(B.EXPORTS)
+    lib = ctypes.CDLL(B._build.LIB)
+    for n in names:
+        assert hasattr(lib, n), f"libdasgd.so does not export {n}"
+
+
+def test_version_and_strerror():
+    assert re.fullmatch(r"\d+\.\d+", B.dasgd_version())
+    assert B._L.dasgd_strerror(B.DASGD_ERR_NO_SLOT) == b"no free snapshot slot"
+
+
+def _cfg(**kw):
+    c = B.dasgd_config()
+    c.K, c.tau, c.d, c.P, c.n_slots, c.xi = 4, 2, 1, 64, 1, 0.25
+    c.w, c.snap, c.mean = 0x1000, 0x2000, 0x3000
+    c.main_stream, c.side_stream = None, 0x10
+    for k, v in kw.items():
+        setattr(c, k, v)
+    return c
+
+
+@pytest.mark.parametrize("bad,frag", [
+    (dict(K=0), "K must"), (dict(P=0), "P must"), (dict(tau=0), "tau must"), (dict(d=-1), "d must"),
+    (dict(xi=1.5), "xi must"), (dict(ld=8), "ld must"), (dict(n_slots=0), "n_slots"),
+    (dict(d=5, n_slots=2), "n_slots"), (dict(w=None), "must not be NULL"), (dict(momentum=0.9), "needs m"),
+    (dict(dtype=1), "needs w_lp"), (dict(dtype=7), "unknown dtype"), (dict(merge_mode=3), "unknown merge_mode"),
+    (dict(w=0x1004), "16-byte"), (dict(side_stream=None), "must differ"),
+])
+def test_init_rejects_bad_configuration_before_touching_cuda(bad, frag):
+    with pytest.raises(B.DasgdError) as e:
+        B.dasgd_init(_cfg(**bad))
+    assert e.value.status == B.DASGD_ERR_INVALID_ARG
+    assert frag in str(e.value)
+
+
+def test_null_context_is_an_error_not_a_crash():
+    for fn in (B._L.dasgd_snapshot, B._L.dasgd_average_async, B._L.dasgd_merge, B._L.dasgd_sync, B._L.dasgd_destroy):
+        assert fn(None) == B.DASGD_ERR_INVALID_ARG
+    assert B._L.dasgd_step(None, None, 0.1) == B.DASGD_ERR_INVALID_ARG
+
+
+def test_wrapper_refuses_to_run_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    with pytest.raises(RuntimeError):
+        B.DaSGD(2, 8, 1, 1, 0.25)

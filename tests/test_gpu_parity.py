@@ -1,0 +1,232 @@
+"""libdasgd (through its C ABI) against the CPU oracle, element by element, on seeded inputs.
+
+Tolerances (float32 path): per teacher-forced step |gpu-cpu| <= 1e-6*(1+|cpu|); after a free-running
+run of 100 steps <= 1e-4*(1+|cpu|).  bf16 mode compares the float32 masters with the same bounds and
+the bfloat16 copy bit for bit against the cast of the GPU's own master.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2006_00441_b200 import inputs
+from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, make_pair, padded_grad, state_of, to_oracle_grad
+
+pytestmark = pytest.mark.gpu
+
+FUSE_SNAP, FUSE_MERGE = 0x2, 0x4
+# f32 vector tile = 256 threads * 4 units * 4 elements = 4096 elements; bf16 tile = 256*2*8 = 4096
+SIZES = [1, 3, 4, 7, 8, 1000, 4096, 3 * 4096 + 1029]
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2006_00441_b200 import binding
+    return binding
+
+
+def grads(seed, t, K, P, std, dtype, ld):
+    g = inputs.grad_block(seed, t, K, P, std, dtype=dtype)
+    return padded_grad(g, ld)
+
+
+# ------------------------------------------------------------------ teacher-forced, one op at a time
+
+@pytest.mark.parametrize("P", SIZES)
+@pytest.mark.parametrize("K,dtype,mom,wd", [(3, 0, 0.9, 1e-2), (1, 0, 0.0, 0.0), (8, 0, 0.0, 1e-3), (4, 1, 0.9, 0.0),
+                                            (5, 1, 0.0, 1e-2), (33, 0, 0.5, 0.0)])
+def test_local_step_teacher_forced(B, P, K, dtype, mom, wd):
+    ld = P if P % 8 == 0 or P < 8 else (P + 7) // 8 * 8
+    w0 = inputs.shared_start(1, P, 0.5).numpy()
+    gpu, cpu = make_pair(B, K, P, 4, 1, 0.25, mom, wd, dtype=dtype, ld=ld, w0=w0)
+    gd = torch.bfloat16 if dtype else torch.float32
+    for t in range(4):
+        # teacher forcing: the GPU starts every step from the oracle's state
+        gpu.set_state(torch.from_numpy(cpu.w), torch.from_numpy(cpu.m) if mom else None)
+        g = grads(3, t, K, P, 0.3, gd, ld)
+        gpu.local_step(g, 0.1)
+        cpu.local_step(to_oracle_grad(g, P), 0.1)
+        w, m = state_of(gpu)
+        assert_close(w, cpu.w, TOL_STEP, f"w t={t}")
+        if mom:
+            assert_close(m, cpu.m, TOL_STEP, f"m t={t}")
+        if dtype:
+            np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), bf16_bits(gpu.w[:, :P].to(torch.bfloat16)))
+        if ld > P:  # padding columns are never touched
+            assert float(gpu.w[:, P:].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("P", SIZES)
+@pytest.mark.parametrize("K,dtype,mode", [(2, 0, 0), (3, 0, 0), (8, 0, 1), (32, 0, 0), (33, 0, 0), (4, 1, 0), (3, 1, 1)])
+def test_snapshot_mean_merge_teacher_forced(B, P, K, dtype, mode):
+    ld = P if P % 8 == 0 or P < 8 else (P + 7) // 8 * 8
+    r = np.random.default_rng(P * 131 + K)
+    W = r.standard_normal((K, P)).astype(np.float32)
+    gpu, cpu = make_pair(B, K, P, 2, 1, 0.25, 0.0, 0.0, dtype=dtype, merge_mode=mode, ld=ld, w0=W)
+    gd = torch.bfloat16 if dtype else torch.float32
+    gpu.snapshot(); gpu.average_async()
+    cpu.snapshot(); cpu.average()
+    gpu.sync()
+    s, snap, mean = cpu.pending(0)
+    np.testing.assert_array_equal(gpu.snap[0, :, :P].cpu().numpy(), snap)           # a copy is exact
+    assert_close(gpu.pending_mean(0).cpu().numpy(), mean, TOL_STEP, "mean")
+    # teacher forcing: hand the oracle's mean to the GPU before the merge
+    gpu.mean[0, :P] = torch.from_numpy(mean).cuda()
+    torch.cuda.synchronize()
+    g = grads(5, 0, K, P, 0.3, gd, ld)
+    gpu.local_step(g, 0.1); cpu.local_step(to_oracle_grad(g, P), 0.1)
+    gpu.set_state(torch.from_numpy(cpu.w))
+    gpu.merge(); cpu.merge()
+    w, _ = state_of(gpu)
+    assert_close(w, cpu.w, TOL_STEP, "merged w")
+    if dtype:
+        np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), bf16_bits(gpu.w[:, :P].to(torch.bfloat16)))
+    assert gpu.n_pending == 0 and cpu.n_pending == 0
+
+
+# ------------------------------------------------------------------ free-running schedules
+
+SCHEDULES = [(1, 1), (2, 1), (4, 1), (1, 2), (2, 2), (4, 2), (2, 3), (3, 0), (1, 0)]
+
+
+@pytest.mark.parametrize("tau,d", SCHEDULES)
+@pytest.mark.parametrize("flags", [0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE])
+@pytest.mark.parametrize("K,dtype,mode", [(4, 0, 0), (3, 1, 0), (8, 0, 1)])
+def test_free_running_100_steps(B, tau, d, flags, K, dtype, mode):
+    P, T = 2 * 4096 + 77, 100
+    ld = (P + 7) // 8 * 8
+    w0 = inputs.shared_start(2, P, 0.02).numpy()
+    gpu, cpu = make_pair(B, K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld, w0=w0)
+    gd = torch.bfloat16 if dtype else torch.float32
+    for t in range(T):
+        g = grads(7, t, K, P, 0.0316, gd, ld)
+        gpu.step(g, 0.1)
+        cpu.step(to_oracle_grad(g, P), 0.1)
+        assert gpu.n_pending == cpu.n_pending
+    w, m = state_of(gpu)
+    assert gpu.t == cpu.t == T
+    assert_close(w, cpu.w, TOL_RUN, "w after 100 steps")
+    assert_close(m, cpu.m, TOL_RUN, "m after 100 steps")
+    if dtype:
+        np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), bf16_bits(gpu.w[:, :P].to(torch.bfloat16)))
+    for i in range(cpu.n_pending):
+        _, _, mean = cpu.pending(i)
+        assert_close(gpu.pending_mean(i).cpu().numpy(), mean, TOL_RUN, f"pending mean {i}")
+
+
+@pytest.mark.parametrize("tau,d", SCHEDULES)
+@pytest.mark.parametrize("dtype,mode", [(0, 0), (1, 0), (0, 1)])
+def test_fused_schedules_are_bit_identical_to_unfused(B, tau, d, dtype, mode):
+    K, P, T = 4, 4096 + 13, 25
+    ld = (P + 7) // 8 * 8
+    w0 = inputs.shared_start(4, P, 0.02)
+    gd = torch.bfloat16 if dtype else torch.float32
+    outs = []
+    for flags in (0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE):
+        gpu = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld)
+        gpu.set_state(w0)
+        for t in range(T):
+            gpu.step(grads(9, t, K, P, 0.0316, gd, ld), 0.1)
+        gpu.sync()
+        outs.append((gpu.w.clone(), gpu.m.clone(), gpu.launches))
+    for w, m, _ in outs[1:]:
+        assert torch.equal(w, outs[0][0]) and torch.equal(m, outs[0][1])
+    if d >= 1:
+        assert outs[1][2] < outs[0][2]  # the fused snapshot removes launches
+
+
+def test_unaligned_rows_and_gradient_pointer_take_the_scalar_path(B):
+    K, P, T = 3, 1001, 12
+    w0 = inputs.shared_start(5, P, 0.1).numpy()
+    gpu, cpu = make_pair(B, K, P, 2, 1, 0.25, 0.9, 1e-3, ld=P, w0=w0)       # ld = 1001: rows not 16-byte aligned
+    for t in range(T):
+        g = grads(11, t, K, P, 0.1, torch.float32, P)
+        gpu.step(g, 0.05); cpu.step(to_oracle_grad(g, P), 0.05)
+    w, m = state_of(gpu)
+    assert_close(w, cpu.w, TOL_RUN); assert_close(m, cpu.m, TOL_RUN)
+    # aligned rows, misaligned gradient base pointer
+    P = 1024
+    gpu, cpu = make_pair(B, K, P, 2, 1, 0.25, 0.9, 0.0, w0=np.zeros(P, np.float32))
+    buf = torch.zeros(K * P + 1, device="cuda")
+    g = buf[1:].view(K, P)
+    g.copy_(inputs.grad_block(12, 0, K, P, 0.1))
+    gpu.step(g, 0.05); cpu.step(to_oracle_grad(g, P), 0.05)
+    w, _ = state_of(gpu)
+    assert_close(w, cpu.w, TOL_STEP)
+
+
+# ------------------------------------------------------------------ explicit call sequence and misuse
+
+def test_explicit_calls_equal_step(B):
+    K, P, tau, d, T = 4, 5000, 2, 1, 9
+    w0 = inputs.shared_start(6, P, 0.1)
+    a = B.DaSGD(K, P, tau, d, 0.25, 0.9)
+    b = B.DaSGD(K, P, tau, d, 0.25, 0.9)
+    a.set_state(w0); b.set_state(w0)
+    for t in range(T):
+        g = grads(13, t, K, P, 0.1, torch.float32, P)
+        a.step(g, 0.1)
+        b.local_step(g, 0.1)
+        u = t + 1
+        if u - d >= tau and (u - d) % tau == 0:
+            b.merge()
+        if u % tau == 0:
+            b.snapshot(); b.average_async()
+    a.sync(); b.sync()
+    assert torch.equal(a.w, b.w) and torch.equal(a.m, b.m)
+
+
+def test_misuse_returns_status_codes(B):
+    gpu = B.DaSGD(2, 64, 2, 1, 0.25)
+    with pytest.raises(B.DasgdError) as e:
+        gpu.merge()
+    assert e.value.status == B.DASGD_ERR_BAD_STATE
+    with pytest.raises(B.DasgdError) as e:
+        gpu.average_async()
+    assert e.value.status == B.DASGD_ERR_BAD_STATE
+    gpu.snapshot()
+    with pytest.raises(B.DasgdError) as e:
+        gpu.snapshot()
+    assert e.value.status == B.DASGD_ERR_NO_SLOT
+    with pytest.raises(B.DasgdError) as e:
+        gpu.merge()                      # snapshot exists but was never averaged
+    assert e.value.status == B.DASGD_ERR_BAD_STATE
+    gpu.average_async(); gpu.merge(); gpu.sync()
+    with pytest.raises(B.DasgdError) as e:
+        gpu.step_host(torch.zeros(2, 64), 0.1)
+    assert e.value.status == B.DASGD_ERR_BAD_STATE
+    # the context is still usable afterwards
+    gpu.step(torch.zeros(2, 64, device="cuda"), 0.1); gpu.sync()
+    assert gpu.t == 1
+
+
+def test_step_host_matches_step(B):
+    K, P, T = 4, 4096 + 8, 6
+    w0 = inputs.shared_start(8, P, 0.1)
+    a = B.DaSGD(K, P, 2, 1, 0.25, 0.9, host_staging=True)
+    b = B.DaSGD(K, P, 2, 1, 0.25, 0.9)
+    a.set_state(w0); b.set_state(w0)
+    probe = torch.empty(256, dtype=torch.float32).pin_memory()
+    hosts = [inputs.grad_block(14, t, K, P, 0.1).pin_memory() for t in range(T)]
+    for t in range(T):
+        a.step_host(hosts[t], 0.1, probe)
+        b.step(hosts[t].cuda(), 0.1)
+    a.sync(); b.sync()
+    assert torch.equal(a.w, b.w)
+    assert torch.equal(probe, a.w[0, :256].cpu())
+
+
+def test_timing_reports_hidden_fraction(B):
+    K, P = 8, 1 << 20
+    gpu = B.DaSGD(K, P, 2, 1, 0.25, 0.9, flags=B.DASGD_FLAG_TIMING)
+    g = torch.zeros(K, P, device="cuda")
+    for _ in range(20):
+        gpu.step(g, 0.1)
+    n, ms_avg, ms_stall = gpu.timing()
+    assert n == 10                     # snapshots (and means) at t = 2, 4, .., 20
+    assert ms_avg > 0 and ms_stall >= 0
+    kt = gpu.kernel_timing()
+    assert kt["local_step"][0] == 20 and kt["snapshot"][0] == 10 and kt["mean"][0] == 10
+    assert kt["merge"][0] == 9 and kt["stall"][0] == 9   # merges at t = 3, 5, .., 19; the last mean stays pending
+    assert all(v[1] > 0 for k, v in kt.items() if k != "stall")
+    gpu.reset_timing()
+    assert gpu.kernel_timing()["local_step"] == (0, 0.0)
