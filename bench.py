@@ -67,7 +67,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", ident, f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", ident, f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -201,7 +201,7 @@ def run_ours(args, wl, name):
         torch.cuda.synchronize()
 
     K, P, lr = wl["K"], wl["P"], wl["lr"]
-    flags_fused = B.DASGD_FLAG_FUSE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE
+    flags_fused = 0 if args.no_fuse else (B.DASGD_FLAG_FUSE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE)
     seed = 1000 + rank  # every rank runs its own replica of the workload
 
     def make(flags, host_staging=False):
@@ -269,6 +269,8 @@ def run_ours(args, wl, name):
     # ---- end to end: gradients start in page-locked host memory every step
     e2e = None
     try:
+        if args.no_e2e:
+            raise RuntimeError("skipped (--no-e2e)")
         eng = make(flags_fused, host_staging=True)
         hosts = [torch.empty((K, P), dtype=torch.float32).pin_memory() for _ in range(2)]
         for i, h in enumerate(hosts):
@@ -295,7 +297,8 @@ def run_ours(args, wl, name):
     if rank != 0:
         return
 
-    cpu = oracle_throughput(wl, seconds_budget=15.0)
+    cpu = (oracle_throughput(wl, seconds_budget=15.0) if not args.no_cpu else
+           {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": "skipped (--no-cpu)"})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -331,14 +334,20 @@ def path_bytes_per_update(wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (profiling on a small case)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    ap.add_argument("--no-fuse", action="store_true", help="run the unfused schedule (separate snapshot copy and merge)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    wl = WORKLOADS[args.workload]
+    wl = dict(WORKLOADS[args.workload])
+    if args.P > 0:
+        wl["P"] = args.P
     if args.impl == "reference":
         run_reference(args, wl, args.workload)
     else:
