@@ -181,6 +181,19 @@ def workload_config(wl, name):
 
 # ------------------------------------------------------------------ our arm
 
+def whole_job(ms_local: float, units_per_rank: float, dist=None, device="cpu"):
+    """Whole-job figures from one rank's device time: the job takes as long as its slowest rank
+    (MAX over ranks) and processes the units of all ranks.  Returns (ms, units/s)."""
+    world = 1
+    ms = float(ms_local)
+    if dist is not None and dist.is_initialized():
+        world = dist.get_world_size()
+        tms = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ms = float(tms.item())
+    return ms, world * units_per_rank / (ms * 1e-3)
+
+
 def run_ours(args, wl, name):
     from paper_2006_00441_b200 import binding as B
 
@@ -229,11 +242,7 @@ def run_ours(args, wl, name):
             ev1.record()
         e.sync()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if dist is not None:
-            tms = torch.tensor([ms], device="cuda")
-            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-            ms = float(tms.item())
+        ms, _ = whole_job(ev0.elapsed_time(ev1), 0.0, dist, "cuda")
         return ms, e.launches - l0
 
     def dev_step(e, t):
