@@ -160,6 +160,30 @@ const char *dasgd_strerror(dasgd_status s);
 const char *dasgd_last_error(const dasgd_ctx *ctx); /* ctx may be NULL: last dasgd_init failure */
 dasgd_status dasgd_destroy(dasgd_ctx *ctx);         /* synchronises both streams, frees the context */
 
+/* Largest P that dasgd_average_merge_noalloc accepts (its built-in mean vector: 4 MiB). */
+#define DASGD_NOALLOC_MAX_P 1048576
+
+/* Averages K replicas and blends the mean back, in one call, WITHOUT any device buffer beyond w:
+ *     mean[p] = (1/K) * sum_k w[k][p];    w[k][p] <- xi*w[k][p] + (1-xi)*mean[p]
+ * i.e. what dasgd_snapshot + dasgd_average_async + dasgd_merge do with d = 0, for callers that
+ * cannot allocate: a serving loop whose device memory pool is frozen once it is warm, a plug-in
+ * that is handed a fixed arena by its host application, a process whose device allocator belongs to
+ * another runtime and must not be bypassed.  (The paper has no counterpart of this call; it is a convenience of this library.)
+ *
+ * w_device: device, [K][ld] float32, in/out (ld = 0 means P).  stream: the cudaStream_t the two kernels
+ * are enqueued on; the call does not wait for them.  device: ordinal of the GPU that holds w.
+ * errbuf (may be NULL): receives a one-line explanation when the status is not DASGD_OK.
+ *
+ * The mean vector is kept in an array built into the library (DASGD_NOALLOC_MAX_P float32 = 4 MiB on
+ * every GPU that loads the library, held until the process exits).  P > DASGD_NOALLOC_MAX_P is refused
+ * with DASGD_ERR_UNSUPPORTED.  The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ * The first call on each device looks up the array's device address; make that first call outside any
+ * stream capture.  All calls on a device share the array: it keeps the previous call's contents, needs no
+ * clearing (every element that is read is overwritten first), and two calls whose kernels can overlap
+ * on the GPU (different streams without ordering between them) race on it -- order them. */
+dasgd_status dasgd_average_merge_noalloc(void *w_device, int32_t K, int64_t P, int64_t ld, float xi,
+                                         int32_t device, void *stream, char *errbuf, int64_t errbuf_len);
+
 /* Library version, "major.minor". */
 const char *dasgd_version(void);
 

@@ -29,6 +29,7 @@ EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
     "dasgd_step", "dasgd_step_host", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
+    "dasgd_average_merge_noalloc",
 ]
 
 
@@ -77,6 +78,7 @@ def _load() -> ctypes.CDLL:
     L.dasgd_last_error.argtypes = [vp]
     L.dasgd_last_error.restype = ctypes.c_char_p
     L.dasgd_destroy.argtypes = [vp]
+    L.dasgd_average_merge_noalloc.argtypes = [vp, i32, i64, i64, f32, i32, vp, ctypes.c_char_p, i64]
     L.dasgd_version.argtypes = []
     L.dasgd_version.restype = ctypes.c_char_p
     return L
@@ -167,6 +169,19 @@ def dasgd_get_launches(ctx) -> int:
 
 def dasgd_destroy(ctx):
     _check(_L.dasgd_destroy(ctx), None)
+
+
+DASGD_NOALLOC_MAX_P = 1 << 20
+
+
+def dasgd_average_merge_noalloc(w_ptr: int, K: int, P: int, ld: int, xi: float, device: int, stream_ptr: int | None):
+    """Average the K rows of w and blend the mean back (xi*w + (1-xi)*mean) using only the library's
+    built-in 4 MiB mean vector: for callers that must not allocate device memory.  P is limited to
+    DASGD_NOALLOC_MAX_P; calls that may overlap on the GPU must be ordered by the caller."""
+    buf = ctypes.create_string_buffer(256)
+    st = _L.dasgd_average_merge_noalloc(w_ptr, K, P, ld, xi, device, stream_ptr, buf, len(buf))
+    if st != DASGD_OK:
+        raise DasgdError(st, f"{_L.dasgd_strerror(st).decode()}: {buf.value.decode()}")
 
 
 # ---------------------------------------------------------------- convenience wrapper

@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdasgd.so")
-SOURCES = [os.path.join(CSRC, "dasgd_api.cu")]
+SOURCES = [os.path.join(CSRC, "dasgd_api.cu"), os.path.join(CSRC, "dasgd_noalloc.cu")]
 HEADERS = [os.path.join(CSRC, "dasgd_kernels.cuh"), os.path.join(ROOT, "include", "dasgd.h")]
 
 
