@@ -160,3 +160,60 @@ class LinearRegression:
             r = X.double() @ w[k].double() - y.double()
             tot += float((r * r).mean()) * 0.5
         return tot / self.K
+
+
+class TeacherMLP:
+    """Regression against a fixed random teacher: K replicas of a bias-free ``layers``-deep MLP
+    (``hidden -> hidden``, ReLU between layers) whose weights live as rows of a ``[K, P]`` array,
+    ``P = layers * hidden**2`` (layer ``l`` of replica ``k`` is ``w[k, l*H*H:(l+1)*H*H].view(H, H)``).
+
+    ``forward_backward`` is the workload's forward/backward pass (batched matmuls, i.e. the GEMM
+    library of the device the tensors live on); it returns the loss per replica and writes the
+    weight gradients, in the layout of the parameters, into ``g_out``.
+    """
+
+    def __init__(self, seed: int, K: int, hidden: int, layers: int = 4, batch: int = 256,
+                 device="cpu", dtype=torch.float32):
+        self.seed, self.K, self.H, self.L, self.B = seed, K, hidden, layers, batch
+        self.P = layers * hidden * hidden
+        self.device, self.dtype = torch.device(device), dtype
+        idx = torch.arange(self.P, dtype=torch.int64, device=self.device)
+        self.teacher = normal_f32(seed, 7, idx, (1.0 / hidden) ** 0.5).to(dtype).view(layers, hidden, hidden)
+
+    def student_init(self) -> torch.Tensor:
+        """Shared start of all replicas, N(0, 2/H), float32 [P]."""
+        idx = torch.arange(self.P, dtype=torch.int64, device=self.device)
+        return normal_f32(self.seed, 8, idx, (2.0 / self.H) ** 0.5)
+
+    def batch_x(self, t: int) -> torch.Tensor:
+        n = self.K * self.B * self.H
+        c = torch.arange(n, dtype=torch.int64, device=self.device) + t * n
+        return normal_f32(self.seed, 9, c, 1.0).to(self.dtype).view(self.K, self.B, self.H)
+
+    def _teacher_out(self, x):
+        h = x
+        for l in range(self.L):
+            h = h @ self.teacher[l].T
+            if l + 1 < self.L:
+                h = torch.relu(h)
+        return h
+
+    def forward_backward(self, t: int, w: torch.Tensor, g_out: torch.Tensor) -> torch.Tensor:
+        """``w``, ``g_out``: ``[K, >=P]`` tensors of ``self.dtype`` (only the first P columns are used)."""
+        K, H, L = self.K, self.H, self.L
+        W = w[:, :self.P].unflatten(1, (L, H, H))          # view, replica stride kept
+        G = g_out[:, :self.P].unflatten(1, (L, H, H))
+        x = self.batch_x(t)
+        y = self._teacher_out(x)
+        acts = [x]
+        for l in range(L):
+            z = torch.bmm(acts[-1], W[:, l].transpose(1, 2))
+            acts.append(torch.relu(z) if l + 1 < L else z)
+        diff = (acts[-1] - y).float()
+        loss = 0.5 * (diff * diff).mean(dim=(1, 2))
+        delta = (diff / (self.B * H)).to(self.dtype)        # d loss / d output
+        for l in reversed(range(L)):
+            G[:, l] = torch.bmm(delta.transpose(1, 2), acts[l])
+            if l > 0:
+                delta = torch.bmm(delta, W[:, l]) * (acts[l] > 0).to(self.dtype)
+        return loss
