@@ -214,7 +214,7 @@ def run_ours(args, wl, name):
         torch.cuda.synchronize()
 
     K, P, lr = wl["K"], wl["P"], wl["lr"]
-    flags_fused = 0 if args.no_fuse else (B.DASGD_FLAG_FUSE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE)
+    flags_fused = 0 if args.no_fuse else (B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE)
     seed = 1000 + rank  # every rank runs its own replica of the workload
 
     def make(flags, host_staging=False):
@@ -330,12 +330,12 @@ def run_ours(args, wl, name):
 
 
 def path_bytes_per_update(wl):
-    """Algorithmic HBM bytes per replica-parameter update of the whole path as scheduled with both
-    fusion flags, float32 + momentum: tau local steps (20 B each), the snapshot stored by the kernel
-    that last writes w (4 B), the mean (4 + 4/K B), and the merge (4/K B inside a step kernel when
-    d >= 2, else a pass of its own: 8 + 4/K B)."""
+    """Algorithmic HBM bytes per replica-parameter update of the whole path as bench.py schedules it
+    (rotating snapshots, merge folded into a step kernel when d >= 2), float32 + momentum: tau local
+    steps (20 B each), the snapshot (0 B: no copy), the mean (4 + 4/K B), and the merge (4/K B inside
+    a step kernel when d >= 2, else a pass of its own: 8 + 4/K B)."""
     K, tau, d = wl["K"], wl["tau"], wl["d"]
-    per_cycle = 20.0 * tau + 4.0 + (4.0 + 4.0 / K)
+    per_cycle = 20.0 * tau + (4.0 + 4.0 / K)
     per_cycle += (4.0 / K) if d >= 2 else (8.0 + 4.0 / K)
     return per_cycle / tau
 

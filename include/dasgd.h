@@ -63,6 +63,13 @@ typedef enum {
 #define DASGD_FLAG_FUSE_MERGE 0x4u    /* dasgd_step: when d >= 2, blend the mean inside the local-step
                                          kernel of the step the merge lands on                         */
 
+#define DASGD_FLAG_ROTATE_SNAPSHOT 0x8u /* snapshots cost no copy: w and the n_slots arrays of snap form a
+                                         pool of n_slots+1 weight arrays; a snapshot freezes the array that
+                                         holds the current weights and the next kernel that writes weights
+                                         writes them into a free array.  The current weights then move
+                                         between arrays: ask dasgd_get_weights where they are.  Results are
+                                         the same as without the flag.  FUSE_SNAPSHOT has no effect.        */
+
 typedef struct dasgd_config {
   int32_t K;            /* workers (the paper's M), >= 1                                              */
   int32_t tau;          /* local steps between snapshots, >= 1                                        */
@@ -79,10 +86,11 @@ typedef struct dasgd_config {
   float momentum;       /* mu; 0 disables the momentum buffer (m may then be NULL)                    */
   float weight_decay;   /* lambda, coupled L2: g' = g + lambda*w                                      */
   uint32_t sync_timeout_ms; /* dasgd_sync gives up after this long; 0 means 60000                     */
-  void *w;              /* device, [K][ld] float32, in/out: weights (master weights in bf16 mode)     */
+  void *w;              /* device, [K][ld] float32, in/out: weights (master weights in bf16 mode); with
+                           DASGD_FLAG_ROTATE_SNAPSHOT: where the weights START (see dasgd_get_weights)  */
   void *m;              /* device, [K][ld] float32, in/out: momentum buffers (start them at 0)        */
   void *w_lp;           /* device, [K][ld] bfloat16, out: low-precision weights; bf16 mode only       */
-  void *snap;           /* device, [n_slots][K][ld] float32, scratch: snapshots                       */
+  void *snap;           /* device, [n_slots][K][ld] float32, scratch: snapshots (ROTATE: weight arrays) */
   void *mean;           /* device, [n_slots][ld] float32, scratch: worker-axis means                  */
   void *g_stage;        /* device, [K][ld] gradient dtype, scratch for dasgd_step_host; may be NULL   */
   void *main_stream;    /* cudaStream_t carrying local steps, snapshots and merges                    */
@@ -130,6 +138,11 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads_device, float lr);
  * asynchronous).  DASGD_ERR_BAD_STATE if cfg.g_stage was NULL. */
 dasgd_status dasgd_step_host(dasgd_ctx *ctx, const void *grads_host, float lr, float *probe_host,
                              int64_t probe_elems);
+
+/* Device pointer of the [K][ld] float32 array that holds the current weights: cfg.w, unless
+ * DASGD_FLAG_ROTATE_SNAPSHOT is set, in which case it can be cfg.w or any of the n_slots arrays of
+ * cfg.snap and is valid until the next call that writes weights (local_step, merge, step). */
+dasgd_status dasgd_get_weights(const dasgd_ctx *ctx, void **w_device);
 
 /* t, the number of completed local steps, and the number of snapshots awaiting their merge. */
 dasgd_status dasgd_get_step(const dasgd_ctx *ctx, int64_t *t, int32_t *pending);

@@ -23,11 +23,11 @@ DASGD_OK, DASGD_ERR_INVALID_ARG, DASGD_ERR_BAD_STATE, DASGD_ERR_NO_SLOT = 0, 1, 
 DASGD_ERR_CUDA, DASGD_ERR_TIMEOUT, DASGD_ERR_UNSUPPORTED = 4, 5, 6
 DASGD_F32, DASGD_BF16_MASTER_F32 = 0, 1
 DASGD_MERGE_XI, DASGD_MERGE_DELTA = 0, 1
-DASGD_FLAG_TIMING, DASGD_FLAG_FUSE_SNAPSHOT, DASGD_FLAG_FUSE_MERGE = 0x1, 0x2, 0x4
+DASGD_FLAG_TIMING, DASGD_FLAG_FUSE_SNAPSHOT, DASGD_FLAG_FUSE_MERGE, DASGD_FLAG_ROTATE_SNAPSHOT = 0x1, 0x2, 0x4, 0x8
 
 EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
-    "dasgd_step", "dasgd_step_host", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
+    "dasgd_step", "dasgd_step_host", "dasgd_get_weights", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
     "dasgd_average_merge_noalloc",
 ]
@@ -67,6 +67,7 @@ def _load() -> ctypes.CDLL:
     L.dasgd_step.argtypes = [vp, vp, f32]
     L.dasgd_step_host.argtypes = [vp, vp, f32, vp, i64]
     L.dasgd_get_step.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i32)]
+    L.dasgd_get_weights.argtypes = [vp, ctypes.POINTER(vp)]
     L.dasgd_get_pending.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(vp), ctypes.POINTER(vp)]
     L.dasgd_get_timing.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double),
                                    ctypes.POINTER(ctypes.c_double)]
@@ -131,6 +132,12 @@ def dasgd_step(ctx, grads_ptr: int, lr: float):
 
 def dasgd_step_host(ctx, grads_host_ptr: int, lr: float, probe_host_ptr: int | None, probe_elems: int):
     _check(_L.dasgd_step_host(ctx, grads_host_ptr, lr, probe_host_ptr, probe_elems), ctx)
+
+
+def dasgd_get_weights(ctx) -> int:
+    w = ctypes.c_void_p()
+    _check(_L.dasgd_get_weights(ctx, ctypes.byref(w)), ctx)
+    return w.value
 
 
 def dasgd_get_step(ctx):
@@ -212,7 +219,7 @@ class DaSGD:
         self.n_slots = n_slots if n_slots is not None else min_slots(tau, d)
         dev = self.device
         self.gdtype = torch.bfloat16 if dtype == DASGD_BF16_MASTER_F32 else torch.float32
-        self.w = torch.zeros((K, self.ld), dtype=torch.float32, device=dev)
+        self._w0 = torch.zeros((K, self.ld), dtype=torch.float32, device=dev)
         self.m = torch.zeros((K, self.ld), dtype=torch.float32, device=dev) if momentum != 0.0 else None
         self.w_lp = torch.zeros((K, self.ld), dtype=torch.bfloat16, device=dev) if dtype == DASGD_BF16_MASTER_F32 else None
         self.snap = torch.empty((self.n_slots, K, self.ld), dtype=torch.float32, device=dev)
@@ -228,7 +235,7 @@ class DaSGD:
         cfg.K, cfg.tau, cfg.d, cfg.dtype, cfg.merge_mode = K, tau, d, dtype, merge_mode
         cfg.n_slots, cfg.flags, cfg.device, cfg.P, cfg.ld = self.n_slots, flags, dev.index or 0, P, self.ld
         cfg.xi, cfg.momentum, cfg.weight_decay, cfg.sync_timeout_ms = xi, momentum, weight_decay, sync_timeout_ms
-        cfg.w = self.w.data_ptr()
+        cfg.w = self._w0.data_ptr()
         cfg.m = self.m.data_ptr() if self.m is not None else None
         cfg.w_lp = self.w_lp.data_ptr() if self.w_lp is not None else None
         cfg.snap, cfg.mean = self.snap.data_ptr(), self.mean.data_ptr()
@@ -239,6 +246,16 @@ class DaSGD:
         self.ctx = dasgd_init(cfg)
 
     # -- state ---------------------------------------------------------------
+    @property
+    def w(self) -> torch.Tensor:
+        """The [K, ld] float32 array that holds the current weights (it moves between arrays when
+        DASGD_FLAG_ROTATE_SNAPSHOT is set; fetch it again after every call that writes weights)."""
+        ptr = dasgd_get_weights(self.ctx)
+        if ptr == self._w0.data_ptr():
+            return self._w0
+        slot = (ptr - self.snap.data_ptr()) // (self.K * self.ld * 4)
+        return self.snap[slot]
+
     def set_state(self, w, m=None):
         """Copy initial weights ([P] shared start or [K, P]) and optionally momentum into the buffers."""
         self.sync()  # work already queued on the library's streams must not race with the copies below

@@ -26,6 +26,7 @@ struct Slot {
   int64_t s = 0;                 // completed local steps when the snapshot was taken
   cudaEvent_t e_snap = nullptr;  // main stream: snapshot written
   cudaEvent_t e_avg = nullptr;   // side stream: mean written
+  int buf = -1;                  // index into ctx->pool of the array that holds this snapshot
 };
 
 // A pair of timing events around one piece of stream work, tagged with what it measures.
@@ -59,6 +60,14 @@ struct dasgd_ctx {
   int epu = 4;       // elements per vector unit
   std::vector<Slot> slots;
   std::deque<int> pending;  // slot indices, oldest snapshot first
+  // Weight-sized arrays: pool[0] = cfg.w, pool[1 + i] = the i-th [K][ld] array of cfg.snap.
+  // `cur` holds the current weights; frozen[b] >= 0 names the pending slot whose snapshot is pool[b].
+  // Copy mode: cur stays 0 and snapshots are copies.  Rotate mode: a snapshot freezes `cur` itself and
+  // the next kernel that writes weights writes them into a free array, which becomes `cur`.
+  std::vector<float *> pool;
+  std::vector<int> frozen;
+  int cur = 0;
+  bool rotate = false;
   std::vector<Span> spans;
   int64_t span_n[TAG_COUNT] = {0, 0, 0, 0, 0};
   double span_ms[TAG_COUNT] = {0, 0, 0, 0, 0};
@@ -84,16 +93,15 @@ dasgd_status cuda_fail(dasgd_ctx *c, cudaError_t e, const char *what) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-float *snap_ptr(const dasgd_ctx *c, int slot) {
-  return static_cast<float *>(c->cfg.snap) + (size_t)slot * c->cfg.K * c->cfg.ld;
-}
+float *snap_ptr(const dasgd_ctx *c, int slot) { return c->pool[c->slots[slot].buf]; }
 float *mean_ptr(const dasgd_ctx *c, int slot) {
   return static_cast<float *>(c->cfg.mean) + (size_t)slot * c->cfg.ld;
 }
 
 Params base_params(const dasgd_ctx *c) {
   Params p{};
-  p.w = static_cast<float *>(c->cfg.w);
+  p.w = c->pool[c->cur];
+  p.w_out = c->pool[c->cur];
   p.m = static_cast<float *>(c->cfg.m);
   p.w_lp = static_cast<__nv_bfloat16 *>(c->cfg.w_lp);
   p.P = c->cfg.P;
@@ -289,12 +297,29 @@ int find_free_slot(const dasgd_ctx *c) {
   return -1;
 }
 
-// book-keeping after the main stream has been given the work that writes snap[slot]
-dasgd_status mark_snapped(dasgd_ctx *c, int slot) {
+// An array that is neither the current weights nor a pending snapshot; `fallback` (or -1) otherwise.
+int find_free_buf(const dasgd_ctx *c, int fallback) {
+  for (size_t b = 0; b < c->pool.size(); ++b)
+    if ((int)b != c->cur && c->frozen[b] < 0) return (int)b;
+  return fallback;
+}
+
+// Where the next kernel that writes weights must put them: in place unless the current array is a
+// pending snapshot.  `reusable` is an array the same kernel is allowed to overwrite element by
+// element after reading it (the snapshot of the slot it merges), or -1.
+int pick_w_out(const dasgd_ctx *c, int reusable) {
+  if (c->frozen[c->cur] < 0) return c->cur;
+  return find_free_buf(c, reusable);
+}
+
+// book-keeping after the main stream has been given the work that completes the snapshot in pool[buf]
+dasgd_status mark_snapped(dasgd_ctx *c, int slot, int buf) {
   Slot &sl = c->slots[slot];
   CU(c, cudaEventRecord(sl.e_snap, c->s0));
   sl.state = SLOT_SNAPPED;
   sl.s = c->t;
+  sl.buf = buf;
+  c->frozen[buf] = slot;
   c->pending.push_back(slot);
   return DASGD_OK;
 }
@@ -309,6 +334,9 @@ dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
   const int sp = span_begin(c, TAG_STALL, c->s0);
   CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg, 0));
   span_end(c, sp, c->s0);
+  // From here on the main stream is ordered after the mean kernel.  The xi-blend no longer needs
+  // the snapshot itself, so its array may be overwritten by what the main stream does next.
+  if (c->cfg.merge_mode == DASGD_MERGE_XI && sl.buf >= 0) c->frozen[sl.buf] = -1;
   *slot_out = slot;
   return DASGD_OK;
 }
@@ -316,7 +344,9 @@ dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
 void release_oldest(dasgd_ctx *c) {
   const int slot = c->pending.front();
   c->pending.pop_front();
-  c->slots[slot].state = SLOT_FREE;
+  Slot &sl = c->slots[slot];
+  if (sl.buf >= 0 && c->frozen[sl.buf] == slot) c->frozen[sl.buf] = -1;
+  sl.state = SLOT_FREE;
 }
 
 bool merge_due(const dasgd_ctx *c, int64_t u) {
@@ -410,6 +440,11 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   ctx->s1 = static_cast<cudaStream_t>(c.side_stream);
   ctx->epu = c.dtype == DASGD_BF16_MASTER_F32 ? 8 : 4;
   ctx->vec = (c.ld % ctx->epu) == 0;
+  ctx->rotate = (c.flags & DASGD_FLAG_ROTATE_SNAPSHOT) != 0;
+  ctx->pool.push_back(static_cast<float *>(c.w));
+  for (int i = 0; i < c.n_slots; ++i)
+    ctx->pool.push_back(static_cast<float *>(c.snap) + (size_t)i * c.K * c.ld);
+  ctx->frozen.assign(ctx->pool.size(), -1);
   DeviceGuard guard(c.device);
   ctx->slots.resize(c.n_slots);
   for (Slot &sl : ctx->slots) {
@@ -444,28 +479,80 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
   return DASGD_OK;
 }
 
+// ---- the four operations, on the pool of weight arrays -------------------------------------------
+
+namespace {
+
+// Local step, optionally with the merge of `merge_slot` (-1: none) folded in and, in copy mode,
+// the snapshot stored into pool[snap_buf] (-1: none).
+dasgd_status op_step(dasgd_ctx *c, const void *grads, float lr, int merge_slot, int snap_buf) {
+  Params p = base_params(c);
+  p.g = grads;
+  p.lr = lr;
+  int reusable = -1;
+  if (merge_slot >= 0) {
+    p.mean = mean_ptr(c, merge_slot);
+    p.snap_in = snap_ptr(c, merge_slot);
+    reusable = c->slots[merge_slot].buf;
+  }
+  const int out = pick_w_out(c, reusable);
+  if (out < 0) return fail(c, DASGD_ERR_NO_SLOT, "step: no free weight array to write into");
+  p.w_out = c->pool[out];
+  if (snap_buf >= 0) p.snap_out = c->pool[snap_buf];
+  const int mode = merge_slot < 0 ? 0 : (c->cfg.merge_mode == DASGD_MERGE_DELTA ? 2 : 1);
+  dasgd_status st = launch_step(c, p, grads_vec_ok(c, grads), mode, snap_buf >= 0);
+  if (st != DASGD_OK) return st;
+  c->cur = out;
+  c->t += 1;
+  return DASGD_OK;
+}
+
+// Stand-alone merge of `slot` (already waited for), optionally storing the snapshot into pool[snap_buf].
+dasgd_status op_merge(dasgd_ctx *c, int slot, int snap_buf) {
+  Params p = base_params(c);
+  p.mean = mean_ptr(c, slot);
+  p.snap_in = snap_ptr(c, slot);
+  const int out = pick_w_out(c, c->slots[slot].buf);
+  if (out < 0) return fail(c, DASGD_ERR_NO_SLOT, "merge: no free weight array to write into");
+  p.w_out = c->pool[out];
+  if (snap_buf >= 0) p.snap_out = c->pool[snap_buf];
+  dasgd_status st = launch_merge(c, p, snap_buf >= 0);
+  if (st != DASGD_OK) return st;
+  c->cur = out;
+  return DASGD_OK;
+}
+
+// Snapshot of the current weights.  Rotate mode: no kernel, the current array is frozen.  Copy mode:
+// `already_in` >= 0 says a fused kernel has stored the copy into pool[already_in]; otherwise copy now.
+dasgd_status op_snapshot(dasgd_ctx *c, int already_in) {
+  const int slot = find_free_slot(c);
+  if (slot < 0) return fail(c, DASGD_ERR_NO_SLOT, "snapshot: every slot holds a pending average");
+  if (c->rotate) return mark_snapped(c, slot, c->cur);
+  int buf = already_in;
+  if (buf < 0) {
+    buf = find_free_buf(c, -1);
+    if (buf < 0) return fail(c, DASGD_ERR_NO_SLOT, "snapshot: no free snapshot array");
+    Params p = base_params(c);
+    p.snap_out = c->pool[buf];
+    dasgd_status st = launch_snapshot(c, p);
+    if (st != DASGD_OK) return st;
+  }
+  return mark_snapped(c, slot, buf);
+}
+
+}  // namespace
+
 dasgd_status dasgd_local_step(dasgd_ctx *ctx, const void *grads, float lr) {
   if (!ctx) return DASGD_ERR_INVALID_ARG;
   if (!grads) return fail(ctx, DASGD_ERR_INVALID_ARG, "local_step: grads is NULL");
   DeviceGuard guard(ctx->cfg.device);
-  Params p = base_params(ctx);
-  p.g = grads;
-  p.lr = lr;
-  dasgd_status st = launch_step(ctx, p, grads_vec_ok(ctx, grads), 0, false);
-  if (st == DASGD_OK) ctx->t += 1;
-  return st;
+  return op_step(ctx, grads, lr, -1, -1);
 }
 
 dasgd_status dasgd_snapshot(dasgd_ctx *ctx) {
   if (!ctx) return DASGD_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->cfg.device);
-  const int slot = find_free_slot(ctx);
-  if (slot < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "snapshot: every slot holds a pending average");
-  Params p = base_params(ctx);
-  p.snap_out = snap_ptr(ctx, slot);
-  dasgd_status st = launch_snapshot(ctx, p);
-  if (st != DASGD_OK) return st;
-  return mark_snapped(ctx, slot);
+  return op_snapshot(ctx, -1);
 }
 
 dasgd_status dasgd_average_async(dasgd_ctx *ctx) {
@@ -480,10 +567,7 @@ dasgd_status dasgd_merge(dasgd_ctx *ctx) {
   int slot = -1;
   dasgd_status st = wait_oldest_average(ctx, &slot);
   if (st != DASGD_OK) return st;
-  Params p = base_params(ctx);
-  p.mean = mean_ptr(ctx, slot);
-  p.snap_in = snap_ptr(ctx, slot);
-  st = launch_merge(ctx, p, false);
+  st = op_merge(ctx, slot, -1);
   if (st != DASGD_OK) return st;
   release_oldest(ctx);
   return DASGD_OK;
@@ -498,63 +582,43 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
   const bool m_due = merge_due(ctx, u);
   const bool s_due = (u % cfg.tau) == 0;
   const bool fuse_merge = m_due && (cfg.flags & DASGD_FLAG_FUSE_MERGE) && cfg.d >= 2;
-  const bool fuse_snap = s_due && (cfg.flags & DASGD_FLAG_FUSE_SNAPSHOT);
-  const int mode = cfg.merge_mode == DASGD_MERGE_DELTA ? 2 : 1;
+  // copy mode only: let the kernel that last writes w in this iteration also store the snapshot
+  const bool fuse_snap = s_due && !ctx->rotate && (cfg.flags & DASGD_FLAG_FUSE_SNAPSHOT);
   dasgd_status st;
-
-  // The snapshot of this iteration may reuse the slot whose mean is merged in this same iteration:
-  // each thread reads the old snapshot/mean elements before it overwrites them.
-  int merge_slot = -1, snap_slot = -1;
-  Params p = base_params(ctx);
-  p.g = grads;
-  p.lr = lr;
+  int stored_in = -1;  // array a fused kernel has stored this iteration's snapshot into
 
   // ---- local step (optionally with the merge and/or the snapshot store folded in)
+  int merge_slot = -1;
   if (fuse_merge) {
     st = wait_oldest_average(ctx, &merge_slot);
     if (st != DASGD_OK) return st;
-    p.mean = mean_ptr(ctx, merge_slot);
-    p.snap_in = snap_ptr(ctx, merge_slot);
   }
-  const bool step_writes_snap = fuse_snap && (!m_due || fuse_merge);
-  if (step_writes_snap) {
-    snap_slot = fuse_merge ? merge_slot : find_free_slot(ctx);
-    if (snap_slot < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot slot");
-    p.snap_out = snap_ptr(ctx, snap_slot);
+  if (fuse_snap && (!m_due || fuse_merge)) {
+    // A kernel that merges a slot may store the new snapshot over that slot's old one: each thread
+    // reads the old element before it writes the new one.
+    stored_in = find_free_buf(ctx, merge_slot >= 0 ? ctx->slots[merge_slot].buf : -1);
+    if (stored_in < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot array");
   }
-  st = launch_step(ctx, p, grads_vec_ok(ctx, grads), fuse_merge ? mode : 0, step_writes_snap);
+  st = op_step(ctx, grads, lr, merge_slot, stored_in);
   if (st != DASGD_OK) return st;
-  ctx->t = u;
   if (fuse_merge) release_oldest(ctx);
 
   // ---- separate merge kernel (d == 1, or fusion off), optionally storing the snapshot
   if (m_due && !fuse_merge) {
     st = wait_oldest_average(ctx, &merge_slot);
     if (st != DASGD_OK) return st;
-    Params q = base_params(ctx);
-    q.mean = mean_ptr(ctx, merge_slot);
-    q.snap_in = snap_ptr(ctx, merge_slot);
     if (fuse_snap) {
-      snap_slot = merge_slot;
-      q.snap_out = snap_ptr(ctx, snap_slot);
+      stored_in = find_free_buf(ctx, ctx->slots[merge_slot].buf);
+      if (stored_in < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot array");
     }
-    st = launch_merge(ctx, q, fuse_snap);
+    st = op_merge(ctx, merge_slot, stored_in);
     if (st != DASGD_OK) return st;
     release_oldest(ctx);
   }
 
   // ---- snapshot and its mean
   if (s_due) {
-    if (snap_slot >= 0) {
-      st = mark_snapped(ctx, snap_slot);
-    } else {
-      const int slot = find_free_slot(ctx);
-      if (slot < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot slot");
-      Params q = base_params(ctx);
-      q.snap_out = snap_ptr(ctx, slot);
-      st = launch_snapshot(ctx, q);
-      if (st == DASGD_OK) st = mark_snapped(ctx, slot);
-    }
+    st = op_snapshot(ctx, stored_in);
     if (st != DASGD_OK) return st;
     st = do_average(ctx);
     if (st != DASGD_OK) return st;
@@ -562,10 +626,7 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
       int slot = -1;
       st = wait_oldest_average(ctx, &slot);
       if (st != DASGD_OK) return st;
-      Params q = base_params(ctx);
-      q.mean = mean_ptr(ctx, slot);
-      q.snap_in = snap_ptr(ctx, slot);
-      st = launch_merge(ctx, q, false);
+      st = op_merge(ctx, slot, -1);
       if (st != DASGD_OK) return st;
       release_oldest(ctx);
     }
@@ -587,8 +648,8 @@ dasgd_status dasgd_step_host(dasgd_ctx *ctx, const void *grads_host, float lr, f
   dasgd_status st = dasgd_step(ctx, ctx->cfg.g_stage, lr);
   if (st != DASGD_OK) return st;
   if (probe_host && probe_elems > 0)
-    CU(ctx, cudaMemcpyAsync(probe_host, ctx->cfg.w, (size_t)probe_elems * sizeof(float), cudaMemcpyDeviceToHost,
-                            ctx->s0));
+    CU(ctx, cudaMemcpyAsync(probe_host, ctx->pool[ctx->cur], (size_t)probe_elems * sizeof(float),
+                            cudaMemcpyDeviceToHost, ctx->s0));
   return DASGD_OK;
 }
 
@@ -614,6 +675,12 @@ dasgd_status dasgd_get_step(const dasgd_ctx *ctx, int64_t *t, int32_t *pending) 
   if (!ctx) return DASGD_ERR_INVALID_ARG;
   if (t) *t = ctx->t;
   if (pending) *pending = (int32_t)ctx->pending.size();
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_weights(const dasgd_ctx *ctx, void **w_device) {
+  if (!ctx || !w_device) return DASGD_ERR_INVALID_ARG;
+  *w_device = ctx->pool[ctx->cur];
   return DASGD_OK;
 }
 

@@ -6,6 +6,10 @@
 // kernel), and small CTAs so that a higher-priority side-stream kernel can take SM slots as they
 // retire.  Tensor cores have no role here (about 0.2 flop per byte).
 //
+// Weights are read from `w` and written to `w_out`; the two may be the same array (in-place) or
+// different ones (the old array then stays intact and serves as the snapshot: no copy is made).
+// Each thread reads every element it owns before it writes it, so in-place use is safe.
+//
 // Arithmetic is float32 with explicit fused multiply-adds, the same expressions in every
 // variant, so that fused and unfused schedules give bit-identical results:
 //     g' = fma(lambda, w, g);  m = fma(mu, m, g');  w = fma(-lr, m, w)        (local step)
@@ -23,7 +27,8 @@ namespace dasgd {
 constexpr int kThreads = 256;
 
 struct Params {
-  float *w;             // [K][ld]
+  const float *w;       // [K][ld] weights to read
+  float *w_out;         // [K][ld] where the new weights go (== w for an in-place update)
   float *m;             // [K][ld] or nullptr
   const void *g;        // [K][ld] float or bf16
   __nv_bfloat16 *w_lp;  // [K][ld] or nullptr
@@ -142,7 +147,7 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
         DASGD_F4_APPLY(w, blend_delta(w.x, a.x, s.x), blend_delta(w.y, a.y, s.y), blend_delta(w.z, a.z, s.z),
                        blend_delta(w.w, a.w, s.w))
       }
-      st_stream(reinterpret_cast<float4 *>(p.w + row + e) + f, w);
+      st_stream(reinterpret_cast<float4 *>(p.w_out + row + e) + f, w);
       if (MOM) st_stream(reinterpret_cast<float4 *>(p.m + row + e) + f, m);
       if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + row + e) + f, w);
       w4[j][f] = w;
@@ -174,7 +179,7 @@ __global__ void __launch_bounds__(kThreads) k_local_step_scalar(const Params p, 
   step_elem<MOM>(w, m, g, p);
   if (MERGE == 1) w = blend_xi(w, p.mean[col], p);
   if (MERGE == 2) w = blend_delta(w, p.mean[col], p.snap_in[i]);
-  p.w[i] = w;
+  p.w_out[i] = w;
   if (MOM) p.m[i] = m;
   if (SNAP) p.snap_out[i] = w;
   if (BF16) p.w_lp[i] = __float2bfloat16_rn(w);
@@ -296,7 +301,7 @@ __global__ void __launch_bounds__(kThreads) k_merge_vec(const Params p) {
           DASGD_F4_APPLY(x, blend_delta(x.x, a[f].x, t.x), blend_delta(x.y, a[f].y, t.y),
                          blend_delta(x.z, a[f].z, t.z), blend_delta(x.w, a[f].w, t.w))
         }
-        st_stream(reinterpret_cast<float4 *>(p.w + off) + f, x);
+        st_stream(reinterpret_cast<float4 *>(p.w_out + off) + f, x);
         if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + off) + f, x);
         w[j][f] = x;
       }
@@ -321,7 +326,7 @@ __global__ void __launch_bounds__(kThreads) k_merge_scalar(const Params p, long 
     const long long i = (long long)k * p.ld + col;
     float w = p.w[i];
     w = (MODE == 1) ? blend_xi(w, a, p) : blend_delta(w, a, p.snap_in[i]);
-    p.w[i] = w;
+    p.w_out[i] = w;
     if (SNAP) p.snap_out[i] = w;
     if (BF16) p.w_lp[i] = __float2bfloat16_rn(w);
   }

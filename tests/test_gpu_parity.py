@@ -13,7 +13,7 @@ from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, make_pair,
 
 pytestmark = pytest.mark.gpu
 
-FUSE_SNAP, FUSE_MERGE = 0x2, 0x4
+FUSE_SNAP, FUSE_MERGE, ROTATE = 0x2, 0x4, 0x8
 # f32 vector tile = 256 threads * 4 units * 4 elements = 4096 elements; bf16 tile = 256*2*8 = 4096
 SIZES = [1, 3, 4, 7, 8, 1000, 4096, 3 * 4096 + 1029]
 
@@ -67,6 +67,8 @@ def test_snapshot_mean_merge_teacher_forced(B, P, K, dtype, mode):
     cpu.snapshot(); cpu.average()
     gpu.sync()
     s, snap, mean = cpu.pending(0)
+    _, snap_ptr, _ = B.dasgd_get_pending(gpu.ctx, 0)
+    assert snap_ptr == gpu.snap[0].data_ptr()
     np.testing.assert_array_equal(gpu.snap[0, :, :P].cpu().numpy(), snap)           # a copy is exact
     assert_close(gpu.pending_mean(0).cpu().numpy(), mean, TOL_STEP, "mean")
     # teacher forcing: hand the oracle's mean to the GPU before the merge
@@ -89,7 +91,7 @@ SCHEDULES = [(1, 1), (2, 1), (4, 1), (1, 2), (2, 2), (4, 2), (2, 3), (3, 0), (1,
 
 
 @pytest.mark.parametrize("tau,d", SCHEDULES)
-@pytest.mark.parametrize("flags", [0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE])
+@pytest.mark.parametrize("flags", [0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE])
 @pytest.mark.parametrize("K,dtype,mode", [(4, 0, 0), (3, 1, 0), (8, 0, 1)])
 def test_free_running_100_steps(B, tau, d, flags, K, dtype, mode):
     P, T = 2 * 4096 + 77, 100
@@ -121,17 +123,18 @@ def test_fused_schedules_are_bit_identical_to_unfused(B, tau, d, dtype, mode):
     w0 = inputs.shared_start(4, P, 0.02)
     gd = torch.bfloat16 if dtype else torch.float32
     outs = []
-    for flags in (0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE):
+    for flags in (0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE):
         gpu = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld)
         gpu.set_state(w0)
         for t in range(T):
             gpu.step(grads(9, t, K, P, 0.0316, gd, ld), 0.1)
         gpu.sync()
-        outs.append((gpu.w.clone(), gpu.m.clone(), gpu.launches))
+        outs.append((gpu.w[:, :P].clone(), gpu.m[:, :P].clone(), gpu.launches))   # payload columns only
     for w, m, _ in outs[1:]:
         assert torch.equal(w, outs[0][0]) and torch.equal(m, outs[0][1])
     if d >= 1:
         assert outs[1][2] < outs[0][2]  # the fused snapshot removes launches
+        assert outs[4][2] < outs[0][2]  # so does the rotating snapshot
 
 
 def test_unaligned_rows_and_gradient_pointer_take_the_scalar_path(B):
@@ -156,11 +159,12 @@ def test_unaligned_rows_and_gradient_pointer_take_the_scalar_path(B):
 
 # ------------------------------------------------------------------ explicit call sequence and misuse
 
-def test_explicit_calls_equal_step(B):
+@pytest.mark.parametrize("flags", [0, ROTATE])
+def test_explicit_calls_equal_step(B, flags):
     K, P, tau, d, T = 4, 5000, 2, 1, 9
     w0 = inputs.shared_start(6, P, 0.1)
-    a = B.DaSGD(K, P, tau, d, 0.25, 0.9)
-    b = B.DaSGD(K, P, tau, d, 0.25, 0.9)
+    a = B.DaSGD(K, P, tau, d, 0.25, 0.9, flags=flags)
+    b = B.DaSGD(K, P, tau, d, 0.25, 0.9, flags=flags)
     a.set_state(w0); b.set_state(w0)
     for t in range(T):
         g = grads(13, t, K, P, 0.1, torch.float32, P)
