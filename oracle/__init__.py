@@ -39,28 +39,33 @@ def build(force: bool = False) -> None:
 _loaded: dict[bool, ctypes.CDLL] = {}
 
 
+def bind(path: str) -> ctypes.CDLL:
+    """Load one build of the oracle and declare its signatures."""
+    L = ctypes.CDLL(path)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    L.oracle_dasgd_create.restype = vp
+    L.oracle_dasgd_create.argtypes = [i32, i64, i32, i32, f32, f32, f32, i32, i32]
+    L.oracle_dasgd_destroy.restype = None
+    L.oracle_dasgd_destroy.argtypes = [vp]
+    L.oracle_dasgd_set_state.argtypes = [vp, vp, vp]
+    L.oracle_dasgd_get_state.argtypes = [vp, vp, vp, vp]
+    L.oracle_dasgd_steps_done.restype = i64
+    L.oracle_dasgd_steps_done.argtypes = [vp]
+    L.oracle_dasgd_pending.argtypes = [vp]
+    L.oracle_dasgd_get_pending.argtypes = [vp, i32, ctypes.POINTER(i64), vp, vp]
+    L.oracle_dasgd_local_step.argtypes = [vp, vp, f32]
+    L.oracle_dasgd_snapshot.argtypes = [vp]
+    L.oracle_dasgd_average.argtypes = [vp]
+    L.oracle_dasgd_merge.argtypes = [vp]
+    L.oracle_dasgd_step.argtypes = [vp, vp, f32]
+    L.oracle_dasgd_threads.argtypes = []
+    return L
+
+
 def _lib(omp: bool) -> ctypes.CDLL:
     if omp not in _loaded:
         build()
-        L = ctypes.CDLL(_LIBS[omp])
-        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
-        L.oracle_dasgd_create.restype = vp
-        L.oracle_dasgd_create.argtypes = [i32, i64, i32, i32, f32, f32, f32, i32, i32]
-        L.oracle_dasgd_destroy.restype = None
-        L.oracle_dasgd_destroy.argtypes = [vp]
-        L.oracle_dasgd_set_state.argtypes = [vp, vp, vp]
-        L.oracle_dasgd_get_state.argtypes = [vp, vp, vp, vp]
-        L.oracle_dasgd_steps_done.restype = i64
-        L.oracle_dasgd_steps_done.argtypes = [vp]
-        L.oracle_dasgd_pending.argtypes = [vp]
-        L.oracle_dasgd_get_pending.argtypes = [vp, i32, ctypes.POINTER(i64), vp, vp]
-        L.oracle_dasgd_local_step.argtypes = [vp, vp, f32]
-        L.oracle_dasgd_snapshot.argtypes = [vp]
-        L.oracle_dasgd_average.argtypes = [vp]
-        L.oracle_dasgd_merge.argtypes = [vp]
-        L.oracle_dasgd_step.argtypes = [vp, vp, f32]
-        L.oracle_dasgd_threads.argtypes = []
-        _loaded[omp] = L
+        _loaded[omp] = bind(_LIBS[omp])
     return _loaded[omp]
 
 
