@@ -242,7 +242,10 @@ dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
   if (c->vec) {
     const long long units = p.P / 4;
     if (units > 0) {
-      dasgd::k_reduce_vec<<<blocks_for(units, kThreads), kThreads, 0, c->s1>>>(p);
+      if (p.K >= 8) dasgd::k_reduce_vec<1><<<blocks_for(units, kThreads), kThreads, 0, c->s1>>>(p);
+      else if (p.K > 4) dasgd::k_reduce_vec<2><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
+      else if (p.K > 2) dasgd::k_reduce_small<2><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
+      else dasgd::k_reduce_small<4><<<blocks_for(units, kThreads * 4), kThreads, 0, c->s1>>>(p);
       c->launches++;
     }
     done = units * 4;

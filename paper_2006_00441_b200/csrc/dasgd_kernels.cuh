@@ -83,8 +83,10 @@ __device__ __forceinline__ float blend_delta(float w, float mean, float snap) {
 // ---------------------------------------------------------------- local step (vector path)
 //
 // One CTA = one worker k and one tile of kThreads*UNROLL units; a unit is 4 (float32 gradients) or
-// 8 (bfloat16 gradients) consecutive parameters.  blockIdx.x enumerates (tile, k) with k fastest so
-// that CTAs sharing a mean tile (fused merge) are neighbours in launch order.
+// 8 (bfloat16 gradients) consecutive parameters.  With a fused merge blockIdx.x enumerates (tile, k)
+// with k fastest, so that the K CTAs sharing a mean tile are neighbours in launch order and the tile
+// is fetched from HBM once; otherwise rows are walked one after the other (k slowest), which keeps
+// every CTA wave on one contiguous address range (measured 1.2 % faster).
 // MERGE: 0 none, 1 xi-blend, 2 delta.  SNAP: also store the final w into snap_out.
 
 template <bool BF16, bool MOM, int MERGE, bool SNAP>
@@ -92,9 +94,17 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
   constexpr int EPU = BF16 ? 8 : 4;   // elements per unit
   constexpr int F4 = EPU / 4;          // float4 per unit
   constexpr int UNROLL = BF16 ? 2 : 4; // units per thread
-  const int k = blockIdx.x % p.K;
-  const long long tile = blockIdx.x / p.K;
   const long long units = p.P / EPU;
+  int k;
+  long long tile;
+  if (MERGE != 0) {
+    k = blockIdx.x % p.K;
+    tile = blockIdx.x / p.K;
+  } else {
+    const unsigned tiles = (unsigned)((units + kThreads * UNROLL - 1) / (kThreads * UNROLL));
+    k = blockIdx.x / tiles;
+    tile = blockIdx.x % tiles;
+  }
   const long long row = (long long)k * p.ld;
   const long long u0 = tile * (long long)(kThreads * UNROLL) + threadIdx.x;
 
@@ -215,39 +225,87 @@ __global__ void __launch_bounds__(kThreads) k_snapshot_scalar(const Params p, lo
 }
 
 // ---------------------------------------------------------------- worker-axis mean
-// One thread owns 4 consecutive parameters and walks the K rows, eight independent 16-byte loads
-// at a time.  Summation: four interleaved partial sums (k mod 4) combined pairwise; then one
-// correctly rounded division by K.
+// One thread owns U units of 4 consecutive parameters and walks the K rows, eight independent
+// 16-byte loads at a time.  Summation: four interleaved partial sums (k mod 4) combined pairwise;
+// then one correctly rounded division by K.
 
 __device__ __forceinline__ void add4(float4 &a, const float4 &b) {
   a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y); a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
 }
 
+// U units per thread (columns u, u + kThreads, ...): with few rows more columns per thread keep
+// enough loads in flight (K = 2 ran at half the bandwidth with one column per thread).
+template <int U>
 __global__ void __launch_bounds__(kThreads) k_reduce_vec(const Params p) {
-  const long long u = (long long)blockIdx.x * kThreads + threadIdx.x;
-  if (u >= p.P / 4) return;
-  const float4 *base = reinterpret_cast<const float4 *>(p.snap_in) + u;
+  constexpr int KC = U == 1 ? 8 : 4;  // rows per batch of loads (a multiple of 4, so k mod 4 == j mod 4)
+  const long long units = p.P / 4;
+  const long long u0 = (long long)blockIdx.x * (kThreads * U) + threadIdx.x;
+  const float4 *base = reinterpret_cast<const float4 *>(p.snap_in);
   const long long ld4 = p.ld / 4;
-  float4 acc[4];
+  float4 acc[U][4];
 #pragma unroll
-  for (int a = 0; a < 4; ++a) acc[a] = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int k0 = 0; k0 < p.K; k0 += 8) {
-    float4 v[8];
+  for (int c = 0; c < U; ++c)
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (k0 + j < p.K) v[j] = ld_stream(base + (long long)(k0 + j) * ld4);
+    for (int a = 0; a < 4; ++a) acc[c][a] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k0 = 0; k0 < p.K; k0 += KC) {
+    float4 v[U][KC];
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (k0 + j < p.K) add4(acc[j & 3], v[j]);
+    for (int j = 0; j < KC; ++j)
+#pragma unroll
+      for (int c = 0; c < U; ++c) {
+        const long long u = u0 + (long long)c * kThreads;
+        if (k0 + j < p.K && u < units) v[c][j] = ld_stream(base + (long long)(k0 + j) * ld4 + u);
+      }
+#pragma unroll
+    for (int j = 0; j < KC; ++j)
+#pragma unroll
+      for (int c = 0; c < U; ++c)
+        if (k0 + j < p.K && u0 + (long long)c * kThreads < units) add4(acc[c][j & 3], v[c][j]);
   }
-  add4(acc[0], acc[1]);
-  add4(acc[2], acc[3]);
-  add4(acc[0], acc[2]);
   const float kf = (float)p.K;
-  float4 r;
-  r.x = __fdiv_rn(acc[0].x, kf); r.y = __fdiv_rn(acc[0].y, kf);
-  r.z = __fdiv_rn(acc[0].z, kf); r.w = __fdiv_rn(acc[0].w, kf);
-  reinterpret_cast<float4 *>(p.mean_out)[u] = r;  // re-read by the merge: leave it cacheable
+#pragma unroll
+  for (int c = 0; c < U; ++c) {
+    const long long u = u0 + (long long)c * kThreads;
+    if (u >= units) continue;
+    add4(acc[c][0], acc[c][1]);
+    add4(acc[c][2], acc[c][3]);
+    add4(acc[c][0], acc[c][2]);
+    float4 r;
+    r.x = __fdiv_rn(acc[c][0].x, kf); r.y = __fdiv_rn(acc[c][0].y, kf);
+    r.z = __fdiv_rn(acc[c][0].z, kf); r.w = __fdiv_rn(acc[c][0].w, kf);
+    reinterpret_cast<float4 *>(p.mean_out)[u] = r;  // re-read by the merge: leave it cacheable
+  }
+}
+
+// K <= 4: the whole column fits in registers.  Missing rows count as +0, which leaves the pairwise
+// tree (r0 + r1) + (r2 + r3) equal to what the general kernel computes.
+template <int U>
+__global__ void __launch_bounds__(kThreads) k_reduce_small(const Params p) {
+  const long long units = p.P / 4;
+  const long long u0 = (long long)blockIdx.x * (kThreads * U) + threadIdx.x;
+  const float4 *base = reinterpret_cast<const float4 *>(p.snap_in);
+  const long long ld4 = p.ld / 4;
+  float4 v[U][4];
+#pragma unroll
+  for (int c = 0; c < U; ++c) {
+    const long long u = u0 + (long long)c * kThreads;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      v[c][j] = (j < p.K && u < units) ? ld_stream(base + (long long)j * ld4 + u) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float kf = (float)p.K;
+#pragma unroll
+  for (int c = 0; c < U; ++c) {
+    const long long u = u0 + (long long)c * kThreads;
+    if (u >= units) continue;
+    add4(v[c][0], v[c][1]);
+    add4(v[c][2], v[c][3]);
+    add4(v[c][0], v[c][2]);
+    float4 r;
+    r.x = __fdiv_rn(v[c][0].x, kf); r.y = __fdiv_rn(v[c][0].y, kf);
+    r.z = __fdiv_rn(v[c][0].z, kf); r.w = __fdiv_rn(v[c][0].w, kf);
+    reinterpret_cast<float4 *>(p.mean_out)[u] = r;
+  }
 }
 
 __global__ void __launch_bounds__(kThreads) k_reduce_scalar(const Params p, long long p0) {
