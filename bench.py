@@ -266,11 +266,31 @@ def run_ours(args, wl, name):
     for t in range(n_inst):
         dev_step(eng, args.warmup + t)
     kt = eng.kernel_timing()
+    # the same kernels with nothing else on the GPU (no side-stream mean beside them)
+    eng.close()
+    del eng
+    eng = make(flags_fused | B.DASGD_FLAG_TIMING)
+    for t in range(3):
+        eng.local_step(ring[t % RING], lr)
+    eng.reset_timing()
+    for t in range(20):
+        eng.local_step(ring[t % RING], lr)
+    eng.sync()
+    for t in range(10):
+        eng.snapshot(); eng.average_async(); eng.sync(); eng.merge(); eng.sync()
+    kt_alone = eng.kernel_timing()
     eng.close()
     del eng
     peak, peak_kind = measured_peak_gbs()
     n_step, ms_step = kt["local_step"]
     step_gbs = (K * P * BYTES_PER_UPDATE_STEP / 1e9) / (ms_step / n_step * 1e-3) if n_step else None
+    alone = {}
+    for kname, nbytes in (("local_step", K * P * BYTES_PER_UPDATE_STEP), ("mean", K * P * 4 + P * 4),
+                          ("merge", K * P * 8 + P * 4)):
+        n_k, ms_k = kt_alone[kname]
+        if n_k:
+            gbs = nbytes / 1e9 / (ms_k / n_k * 1e-3)
+            alone[kname] = {"ms": ms_k / n_k, "GB/s": gbs, "frac": gbs / peak}
     hidden = None
     if kt["mean"][0] and kt["mean"][1] > 0:
         hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
@@ -280,7 +300,7 @@ def run_ours(args, wl, name):
     try:
         if args.no_e2e:
             raise RuntimeError("skipped (--no-e2e)")
-        eng = make(flags_fused, host_staging=True)
+        eng = make(flags_fused, host_staging=2)
         hosts = [torch.empty((K, P), dtype=torch.float32).pin_memory() for _ in range(2)]
         for i, h in enumerate(hosts):
             h.copy_(ring[i])
@@ -319,8 +339,10 @@ def run_ours(args, wl, name):
                      "frac_of_8TBs": (step_gbs / 8000.0) if step_gbs else None,
                      "algorithmic_bytes_per_launch": K * P * BYTES_PER_UPDATE_STEP,
                      "avg_launch_ms": (ms_step / n_step) if n_step else None,
-                     "timed": f"CUDA events on the launching stream, instrumented pass of {n_inst} steps",
-                     "traffic": None},
+                     "timed": f"CUDA events on the launching stream, instrumented pass of {n_inst} steps; the "
+                              "side-stream mean kernel runs beside this kernel and shares HBM with it",
+                     "traffic": None,
+                     "alone": alone},
         "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
         "averaging_hidden_frac": hidden,
         "whole_path_gbs": value / world * path_bytes_per_update(wl) / 1e9,

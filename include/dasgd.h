@@ -14,7 +14,8 @@
  *   - Every pointer named "device" is a CUDA device pointer on the context's device; every
  *     pointer named "host" is ordinary (preferably page-locked) host memory.
  *   - All device buffers and both streams are owned by the caller and must stay valid until
- *     dasgd_destroy().  The library owns only its host-side context and its CUDA events.
+ *     dasgd_destroy().  The library owns only its host-side context, its CUDA events and, when
+ *     gradient staging is configured, one copy stream.
  *   - All calls are asynchronous with respect to the host except dasgd_sync, dasgd_get_timing
  *     and dasgd_destroy.  A context is not thread-safe; different contexts are independent.
  *   - Every call returns a dasgd_status and never aborts.  After a non-OK status
@@ -86,13 +87,16 @@ typedef struct dasgd_config {
   float momentum;       /* mu; 0 disables the momentum buffer (m may then be NULL)                    */
   float weight_decay;   /* lambda, coupled L2: g' = g + lambda*w                                      */
   uint32_t sync_timeout_ms; /* dasgd_sync gives up after this long; 0 means 60000                     */
+  int32_t n_stage;      /* gradient staging arrays behind g_stage: 0 (none), 1, or 2 (the copy of the
+                           next step's gradients then overlaps this step's kernels)                   */
+  int32_t reserved;     /* set to 0                                                                   */
   void *w;              /* device, [K][ld] float32, in/out: weights (master weights in bf16 mode); with
                            DASGD_FLAG_ROTATE_SNAPSHOT: where the weights START (see dasgd_get_weights)  */
   void *m;              /* device, [K][ld] float32, in/out: momentum buffers (start them at 0)        */
   void *w_lp;           /* device, [K][ld] bfloat16, out: low-precision weights; bf16 mode only       */
   void *snap;           /* device, [n_slots][K][ld] float32, scratch: snapshots (ROTATE: weight arrays) */
   void *mean;           /* device, [n_slots][ld] float32, scratch: worker-axis means                  */
-  void *g_stage;        /* device, [K][ld] gradient dtype, scratch for dasgd_step_host; may be NULL   */
+  void *g_stage;        /* device, [n_stage][K][ld] gradient dtype, scratch for dasgd_step_host; may be NULL */
   void *main_stream;    /* cudaStream_t carrying local steps, snapshots and merges                    */
   void *side_stream;    /* cudaStream_t carrying the averages; must differ from main_stream           */
 } dasgd_config;
@@ -132,10 +136,12 @@ dasgd_status dasgd_sync(dasgd_ctx *ctx);
 dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads_device, float lr);
 
 /* dasgd_step for callers whose gradients are in HOST memory: copies grads_host ([K][ld], gradient
- * dtype) into cfg.g_stage on the main stream, runs dasgd_step, and, if probe_host != NULL, copies
- * the first probe_elems float32 weights of worker 0 back into probe_host.  Both host buffers must
- * stay valid until the main stream has passed this call (page-locked memory keeps the copies
- * asynchronous).  DASGD_ERR_BAD_STATE if cfg.g_stage was NULL. */
+ * dtype) into the next staging array of cfg.g_stage on a copy stream owned by the library, makes the
+ * main stream wait for that copy, runs dasgd_step on it and, if probe_host != NULL, copies the first
+ * probe_elems float32 weights of worker 0 back into probe_host on the main stream.  With n_stage = 2
+ * the copy for call i+1 runs while the kernels of call i do.  Both host buffers must stay valid until
+ * dasgd_sync returns (page-locked memory keeps the copies asynchronous).  DASGD_ERR_BAD_STATE if
+ * cfg.g_stage was NULL or n_stage < 1. */
 dasgd_status dasgd_step_host(dasgd_ctx *ctx, const void *grads_host, float lr, float *probe_host,
                              int64_t probe_elems);
 

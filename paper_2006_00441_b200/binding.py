@@ -39,7 +39,7 @@ class dasgd_config(ctypes.Structure):
         ("merge_mode", ctypes.c_int32), ("n_slots", ctypes.c_int32), ("flags", ctypes.c_uint32),
         ("device", ctypes.c_int32), ("P", ctypes.c_int64), ("ld", ctypes.c_int64),
         ("xi", ctypes.c_float), ("momentum", ctypes.c_float), ("weight_decay", ctypes.c_float),
-        ("sync_timeout_ms", ctypes.c_uint32),
+        ("sync_timeout_ms", ctypes.c_uint32), ("n_stage", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("w", ctypes.c_void_p), ("m", ctypes.c_void_p), ("w_lp", ctypes.c_void_p), ("snap", ctypes.c_void_p),
         ("mean", ctypes.c_void_p), ("g_stage", ctypes.c_void_p),
         ("main_stream", ctypes.c_void_p), ("side_stream", ctypes.c_void_p),
@@ -224,7 +224,8 @@ class DaSGD:
         self.w_lp = torch.zeros((K, self.ld), dtype=torch.bfloat16, device=dev) if dtype == DASGD_BF16_MASTER_F32 else None
         self.snap = torch.empty((self.n_slots, K, self.ld), dtype=torch.float32, device=dev)
         self.mean = torch.empty((self.n_slots, self.ld), dtype=torch.float32, device=dev)
-        self.g_stage = torch.empty((K, self.ld), dtype=self.gdtype, device=dev) if host_staging else None
+        n_stage = int(host_staging) if host_staging in (0, 1, 2, True, False) else 0
+        self.g_stage = torch.empty((n_stage, K, self.ld), dtype=self.gdtype, device=dev) if n_stage else None
         try:
             lo, hi = torch.cuda.Stream.priority_range()  # (least, greatest) priority
         except Exception:
@@ -240,6 +241,7 @@ class DaSGD:
         cfg.w_lp = self.w_lp.data_ptr() if self.w_lp is not None else None
         cfg.snap, cfg.mean = self.snap.data_ptr(), self.mean.data_ptr()
         cfg.g_stage = self.g_stage.data_ptr() if self.g_stage is not None else None
+        cfg.n_stage = n_stage
         cfg.main_stream, cfg.side_stream = self.main.cuda_stream, self.side.cuda_stream
         self.cfg = cfg
         torch.cuda.synchronize(dev)  # the zero fills above ran on torch's current stream

@@ -68,6 +68,12 @@ struct dasgd_ctx {
   std::vector<int> frozen;
   int cur = 0;
   bool rotate = false;
+  // host-gradient staging (dasgd_step_host): a copy stream and, per staging array, an event for
+  // "copy landed" (copy stream) and one for "kernels have consumed it" (main stream)
+  cudaStream_t s_copy = nullptr;
+  std::vector<cudaEvent_t> e_copied, e_consumed;
+  std::vector<bool> stage_used;
+  int64_t host_calls = 0;
   std::vector<Span> spans;
   int64_t span_n[TAG_COUNT] = {0, 0, 0, 0, 0};
   double span_ms[TAG_COUNT] = {0, 0, 0, 0, 0};
@@ -430,6 +436,9 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   if (c.main_stream == c.side_stream)
     return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: main_stream and side_stream must differ");
   if (c.sync_timeout_ms == 0) c.sync_timeout_ms = 60000;
+  if (c.n_stage < 0 || c.n_stage > 2) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: n_stage must be 0, 1 or 2");
+  if ((c.n_stage > 0) != (c.g_stage != nullptr))
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: g_stage and n_stage must be given together");
 
   int ndev = 0;
   cudaError_t e = cudaGetDeviceCount(&ndev);
@@ -462,6 +471,19 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
       return st;
     }
   }
+  if (c.n_stage > 0) {
+    bool ok = cudaStreamCreateWithFlags(&ctx->s_copy, cudaStreamNonBlocking) == cudaSuccess;
+    ctx->e_copied.assign(c.n_stage, nullptr);
+    ctx->e_consumed.assign(c.n_stage, nullptr);
+    ctx->stage_used.assign(c.n_stage, false);
+    for (int i = 0; ok && i < c.n_stage; ++i)
+      ok = cudaEventCreateWithFlags(&ctx->e_copied[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->e_consumed[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      dasgd_destroy(ctx);
+      return fail(nullptr, DASGD_ERR_CUDA, "init: cannot create the staging stream and events");
+    }
+  }
   *out = ctx;
   return DASGD_OK;
 }
@@ -478,6 +500,12 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
   for (Span &sp : ctx->spans)
     for (int j = 0; j < 2; ++j)
       if (sp.ev[j]) cudaEventDestroy(sp.ev[j]);
+  if (ctx->s_copy) {
+    cudaStreamSynchronize(ctx->s_copy);
+    cudaStreamDestroy(ctx->s_copy);
+  }
+  for (cudaEvent_t e : ctx->e_copied) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->e_consumed) if (e) cudaEventDestroy(e);
   delete ctx;
   return DASGD_OK;
 }
@@ -641,15 +669,25 @@ dasgd_status dasgd_step_host(dasgd_ctx *ctx, const void *grads_host, float lr, f
                              int64_t probe_elems) {
   if (!ctx) return DASGD_ERR_INVALID_ARG;
   if (!grads_host) return fail(ctx, DASGD_ERR_INVALID_ARG, "step_host: grads_host is NULL");
-  if (!ctx->cfg.g_stage) return fail(ctx, DASGD_ERR_BAD_STATE, "step_host: cfg.g_stage was NULL");
+  if (!ctx->cfg.g_stage || ctx->cfg.n_stage < 1)
+    return fail(ctx, DASGD_ERR_BAD_STATE, "step_host: no gradient staging configured (g_stage, n_stage)");
   if (probe_host && (probe_elems < 0 || probe_elems > ctx->cfg.P))
     return fail(ctx, DASGD_ERR_INVALID_ARG, "step_host: probe_elems must be in [0, P]");
   DeviceGuard guard(ctx->cfg.device);
   const size_t esz = ctx->cfg.dtype == DASGD_BF16_MASTER_F32 ? 2 : 4;
   const size_t bytes = (size_t)ctx->cfg.K * ctx->cfg.ld * esz;
-  CU(ctx, cudaMemcpyAsync(ctx->cfg.g_stage, grads_host, bytes, cudaMemcpyHostToDevice, ctx->s0));
-  dasgd_status st = dasgd_step(ctx, ctx->cfg.g_stage, lr);
+  const int i = (int)(ctx->host_calls % ctx->cfg.n_stage);
+  char *stage = static_cast<char *>(ctx->cfg.g_stage) + (size_t)i * bytes;
+  // the staging array may be overwritten only after the kernels of its previous use have run
+  if (ctx->stage_used[i]) CU(ctx, cudaStreamWaitEvent(ctx->s_copy, ctx->e_consumed[i], 0));
+  CU(ctx, cudaMemcpyAsync(stage, grads_host, bytes, cudaMemcpyHostToDevice, ctx->s_copy));
+  CU(ctx, cudaEventRecord(ctx->e_copied[i], ctx->s_copy));
+  CU(ctx, cudaStreamWaitEvent(ctx->s0, ctx->e_copied[i], 0));
+  dasgd_status st = dasgd_step(ctx, stage, lr);
   if (st != DASGD_OK) return st;
+  CU(ctx, cudaEventRecord(ctx->e_consumed[i], ctx->s0));
+  ctx->stage_used[i] = true;
+  ctx->host_calls += 1;
   if (probe_host && probe_elems > 0)
     CU(ctx, cudaMemcpyAsync(probe_host, ctx->pool[ctx->cur], (size_t)probe_elems * sizeof(float),
                             cudaMemcpyDeviceToHost, ctx->s0));
@@ -660,7 +698,8 @@ dasgd_status dasgd_sync(dasgd_ctx *ctx) {
   if (!ctx) return DASGD_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->cfg.device);
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(ctx->cfg.sync_timeout_ms);
-  cudaStream_t streams[2] = {ctx->s0, ctx->s1};
+  std::vector<cudaStream_t> streams = {ctx->s0, ctx->s1};
+  if (ctx->s_copy) streams.push_back(ctx->s_copy);
   for (cudaStream_t s : streams) {
     for (;;) {
       cudaError_t e = cudaStreamQuery(s);

@@ -44,7 +44,8 @@ def _cfg(**kw):
     (dict(xi=1.5), "xi must"), (dict(ld=8), "ld must"), (dict(n_slots=0), "n_slots"),
     (dict(d=5, n_slots=2), "n_slots"), (dict(w=None), "must not be NULL"), (dict(momentum=0.9), "needs m"),
     (dict(dtype=1), "needs w_lp"), (dict(dtype=7), "unknown dtype"), (dict(merge_mode=3), "unknown merge_mode"),
-    (dict(w=0x1004), "16-byte"), (dict(side_stream=None), "must differ"),
+    (dict(w=0x1004), "16-byte"), (dict(side_stream=None), "must differ"), (dict(n_stage=3, g_stage=0x4000), "n_stage"),
+    (dict(n_stage=1), "given together"), (dict(g_stage=0x4000), "given together"),
 ])
 def test_init_rejects_bad_configuration_before_touching_cuda(bad, frag):
     with pytest.raises(B.DasgdError) as e:
