@@ -36,11 +36,20 @@ WORKLOADS = {
                      g_std=1e-3 ** 0.5, w_std=0.02),
     "small": dict(K=4, P=1024, momentum=0.0, weight_decay=0.0, lr=0.01, tau=4, d=1, xi=0.25,
                   g_std=1.0, w_std=0.0),
+    # BERT-large-sized: bfloat16 gradients and weight copy, float32 master weights / momentum
+    "bert_large": dict(K=4, P=335_000_000, momentum=0.9, weight_decay=0.0, lr=1e-3, tau=2, d=1, xi=0.25,
+                       g_std=1e-2, w_std=0.02, bf16=True, ring=2),
 }
 METRIC = "replica-param updates/s"
 UNIT = "updates/s"
-RING = 4                       # gradient buffers resident in HBM, used round-robin
-BYTES_PER_UPDATE_STEP = 20     # local step, float32 + momentum: read w, m, g; write w, m
+
+
+def step_bytes(wl):
+    """Algorithmic HBM bytes per replica-parameter of one local-step launch."""
+    if wl.get("bf16"):
+        return (2 + 4 + 4 + 4 + 4 + 2) if wl["momentum"] else (2 + 4 + 4 + 2)
+    return 20 if wl["momentum"] else 12   # read w, (m,) g; write w (, m)
+
 
 
 def measured_peak_gbs():
@@ -120,9 +129,16 @@ def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmu
     probe.close()
     # calibrate on a slice too large for the CPU caches, so the rate is the DRAM-bound one
     Pc = min(wl["P"], 2_000_000)
-    o = oracle.OracleDaSGD(K, Pc, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], omp=True)
+    odt = 1 if wl.get("bf16") else 0
+
+    def host_grad(t, idx):
+        g = inputs.grad_block(0, t, K, wl["P"], wl["g_std"], p_index=idx,
+                              dtype=torch.bfloat16 if odt else torch.float32)
+        return g.view(torch.int16).numpy().view(np.uint16) if odt else g.numpy()
+
+    o = oracle.OracleDaSGD(K, Pc, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], dtype=odt, omp=True)
     o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=range(Pc)).numpy())
-    g = inputs.grad_block(0, 0, K, wl["P"], wl["g_std"], p_index=range(Pc)).numpy()
+    g = host_grad(0, range(Pc))
     for _ in range(2):
         o.step(g, wl["lr"])
     t0 = time.perf_counter()
@@ -137,9 +153,9 @@ def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmu
     else:                   # reference arm: the caller fixes the steps, the slice is sized to the budget
         Ps = int(min(wl["P"], 4_000_000, max(1024, seconds_budget * rate / (K * (steps + warmup)))))
     idx = range(Ps)
-    o = oracle.OracleDaSGD(K, Ps, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], omp=True)
+    o = oracle.OracleDaSGD(K, Ps, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], dtype=odt, omp=True)
     o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=idx).numpy())
-    ring = [inputs.grad_block(0, t, K, wl["P"], wl["g_std"], p_index=idx).numpy() for t in range(2)]
+    ring = [host_grad(t, idx) for t in range(2)]
     for t in range(warmup):
         o.step(ring[t % 2], wl["lr"])
     t0 = time.perf_counter()
@@ -162,7 +178,8 @@ def run_reference(args, wl, name):
     line = {
         "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * r["seconds"] / r["steps"],
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 gradients, f32 state" if wl.get("bf16") else "f32", "data": "synthetic",
         "config": workload_config(wl, name),
         "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -172,10 +189,10 @@ def run_reference(args, wl, name):
 
 
 def workload_config(wl, name):
-    return {"workload": f"{name}: K={wl['K']} replicas x P={wl['P']} float32, momentum {wl['momentum']}, "
+    return {"workload": f"{name}: K={wl['K']} replicas x P={wl['P']} {'bf16 gradients + f32 master' if wl.get('bf16') else 'float32'}, momentum {wl['momentum']}, "
                         f"weight decay {wl['weight_decay']}, lr {wl['lr']}, tau={wl['tau']}, d={wl['d']}, xi={wl['xi']}",
             "K": wl["K"], "P": wl["P"], "tau": wl["tau"], "d": wl["d"], "xi": wl["xi"],
-            "l2_policy": "inputs larger than L2 (each step streams K*P*20 B; gradient ring of 4 buffers)",
+            "l2_policy": "inputs larger than L2 (every step streams all K*P-sized arrays; gradients come from a ring of buffers)",
             "parallelism": "independent replicas of the workload per GPU (no collective on this path)"}
 
 
@@ -214,16 +231,20 @@ def run_ours(args, wl, name):
         torch.cuda.synchronize()
 
     K, P, lr = wl["K"], wl["P"], wl["lr"]
+    bf16 = bool(wl.get("bf16"))
+    gdt = torch.bfloat16 if bf16 else torch.float32
+    RING = wl.get("ring", 4)
     flags_fused = 0 if args.no_fuse else (B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE)
     seed = 1000 + rank  # every rank runs its own replica of the workload
 
     def make(flags, host_staging=False):
         e = B.DaSGD(K, P, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], flags=flags,
+                    dtype=B.DASGD_BF16_MASTER_F32 if bf16 else B.DASGD_F32,
                     device=local_rank, host_staging=host_staging, order_after_current=False)
         e.set_state(inputs.shared_start(seed, P, wl["w_std"], device="cuda"))
         return e
 
-    ring = [inputs.grad_block(seed, t, K, P, wl["g_std"], device="cuda") for t in range(RING)]
+    ring = [inputs.grad_block(seed, t, K, P, wl["g_std"], device="cuda", dtype=gdt) for t in range(RING)]
     torch.cuda.synchronize()
 
     def timed_loop(e, steps, warmup, step_fn):
@@ -283,10 +304,10 @@ def run_ours(args, wl, name):
     del eng
     peak, peak_kind = measured_peak_gbs()
     n_step, ms_step = kt["local_step"]
-    step_gbs = (K * P * BYTES_PER_UPDATE_STEP / 1e9) / (ms_step / n_step * 1e-3) if n_step else None
+    step_gbs = (K * P * step_bytes(wl) / 1e9) / (ms_step / n_step * 1e-3) if n_step else None
     alone = {}
-    for kname, nbytes in (("local_step", K * P * BYTES_PER_UPDATE_STEP), ("mean", K * P * 4 + P * 4),
-                          ("merge", K * P * 8 + P * 4)):
+    for kname, nbytes in (("local_step", K * P * step_bytes(wl)), ("mean", K * P * 4 + P * 4),
+                          ("merge", K * P * (10 if bf16 else 8) + P * 4)):
         n_k, ms_k = kt_alone[kname]
         if n_k:
             gbs = nbytes / 1e9 / (ms_k / n_k * 1e-3)
@@ -301,7 +322,7 @@ def run_ours(args, wl, name):
         if args.no_e2e:
             raise RuntimeError("skipped (--no-e2e)")
         eng = make(flags_fused, host_staging=2)
-        hosts = [torch.empty((K, P), dtype=torch.float32).pin_memory() for _ in range(2)]
+        hosts = [torch.empty((K, P), dtype=gdt).pin_memory() for _ in range(2)]
         for i, h in enumerate(hosts):
             h.copy_(ring[i])
         probe = torch.empty(1024, dtype=torch.float32).pin_memory()
@@ -313,7 +334,7 @@ def run_ours(args, wl, name):
 
         ms_e, _ = timed_loop(eng, e2e_steps, 3, host_step)
         e2e = {"value": world * K * P * e2e_steps / (ms_e * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": K * P * 4, "d2h_bytes_per_step": probe.numel() * 4,
+               "h2d_bytes_per_step": K * P * (2 if bf16 else 4), "d2h_bytes_per_step": probe.numel() * 4,
                "steps": e2e_steps, "ms_per_step": ms_e / e2e_steps}
         eng.close()
         del eng, hosts
@@ -323,21 +344,24 @@ def run_ours(args, wl, name):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+    del ring
+    torch.cuda.empty_cache()
     if rank != 0:
-        return
+        return None
 
     cpu = (oracle_throughput(wl, seconds_budget=15.0) if not args.no_cpu else
            {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": "skipped (--no-cpu)"})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": workload_config(wl, name),
+        "dtype": "bf16 gradients, f32 state" if bf16 else "f32", "data": "synthetic", "config": workload_config(wl, name),
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "k_local_step_vec (float32, momentum)",
+        "roofline": {"bound": "hbm", "kernel": "k_local_step_vec (%s%s)" % ("bf16 gradients + f32 master" if bf16 else "float32",
+                                                                ", momentum" if wl["momentum"] else ""),
                      "achieved": step_gbs, "peak": peak, "unit": "GB/s",
                      "frac": (step_gbs / peak) if step_gbs else None, "peak_kind": f"of {peak_kind}",
                      "frac_of_8TBs": (step_gbs / 8000.0) if step_gbs else None,
-                     "algorithmic_bytes_per_launch": K * P * BYTES_PER_UPDATE_STEP,
+                     "algorithmic_bytes_per_launch": K * P * step_bytes(wl),
                      "avg_launch_ms": (ms_step / n_step) if n_step else None,
                      "timed": f"CUDA events on the launching stream, instrumented pass of {n_inst} steps; the "
                               "side-stream mean kernel runs beside this kernel and shares HBM with it",
@@ -348,17 +372,32 @@ def run_ours(args, wl, name):
         "whole_path_gbs": value / world * path_bytes_per_update(wl) / 1e9,
         "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
     }
-    print(json.dumps(line), flush=True)
+    return line
+
+
+def run_sweep(args):
+    """The K x tau x d sweep at P = 25.6M float32 (one JSON line per point), then the bf16 workload."""
+    args.no_e2e = args.no_cpu = True
+    for K in (2, 4, 8, 16, 32):
+        for tau in (1, 2, 4):
+            for d in (1, 2):
+                wl = dict(WORKLOADS["resnet50"], K=K, tau=tau, d=d, weight_decay=0.0)
+                line = run_ours(args, wl, "sweep")
+                if line:
+                    keep = {k: line[k] for k in ("value", "ms_per_step", "gpu_launches", "averaging_hidden_frac",
+                                                 "whole_path_gbs", "kernels_ms_per_launch")}
+                    keep.update(K=K, tau=tau, d=d, local_step_alone_gbs=line["roofline"]["alone"]["local_step"]["GB/s"])
+                    print(json.dumps(keep), flush=True)
 
 
 def path_bytes_per_update(wl):
     """Algorithmic HBM bytes per replica-parameter update of the whole path as bench.py schedules it
-    (rotating snapshots, merge folded into a step kernel when d >= 2), float32 + momentum: tau local
-    steps (20 B each), the snapshot (0 B: no copy), the mean (4 + 4/K B), and the merge (4/K B inside
-    a step kernel when d >= 2, else a pass of its own: 8 + 4/K B)."""
+    (rotating snapshots, merge folded into a step kernel when d >= 2): tau local steps, the snapshot
+    (0 B: no copy), the mean (4 + 4/K B), and the merge (4/K B inside a step kernel when d >= 2, else a
+    pass of its own: 8 + 4/K B, + 2 B for the bfloat16 copy)."""
     K, tau, d = wl["K"], wl["tau"], wl["d"]
-    per_cycle = 20.0 * tau + (4.0 + 4.0 / K)
-    per_cycle += (4.0 / K) if d >= 2 else (8.0 + 4.0 / K)
+    per_cycle = step_bytes(wl) * tau + (4.0 + 4.0 / K)
+    per_cycle += (4.0 / K) if d >= 2 else (8.0 + 4.0 / K + (2.0 if wl.get("bf16") else 0.0))
     return per_cycle / tau
 
 
@@ -370,19 +409,33 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (profiling on a small case)")
+    ap.add_argument("--K", type=int, default=0, help="override the number of replicas (sweep)")
+    ap.add_argument("--tau", type=int, default=0, help="override the averaging period (sweep)")
+    ap.add_argument("--d", type=int, default=-1, help="override the delay (sweep)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-fuse", action="store_true", help="run the unfused schedule (separate snapshot copy and merge)")
+    ap.add_argument("--sweep", action="store_true", help="run the K x tau x d sweep instead (one JSON line per point)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     wl = dict(WORKLOADS[args.workload])
     if args.P > 0:
         wl["P"] = args.P
-    if args.impl == "reference":
+    if args.K > 0:
+        wl["K"] = args.K
+    if args.tau > 0:
+        wl["tau"] = args.tau
+    if args.d >= 0:
+        wl["d"] = args.d
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, wl, args.workload)
     else:
-        run_ours(args, wl, args.workload)
+        line = run_ours(args, wl, args.workload)
+        if line:
+            print(json.dumps(line), flush=True)
 
 
 if __name__ == "__main__":
