@@ -172,6 +172,20 @@ dasgd_status dasgd_get_kernel_timing(dasgd_ctx *ctx, int32_t which, int64_t *n, 
 /* Synchronises and zeroes every timing counter. */
 dasgd_status dasgd_reset_timing(dasgd_ctx *ctx);
 
+/* Delay guideline of Section III-D (Eq. 3) and Section VI-C/VI-D: the averaging is fully hidden when
+ * t_c < d * t_p (t_c: time of one averaging, t_p: time of one local update, same unit), so *d is the
+ * smallest positive integer with that property and *tau = *d + 1.  Pure host arithmetic.
+ * DASGD_ERR_INVALID_ARG unless t_c >= 0, t_p > 0 and both outputs are non-NULL. */
+dasgd_status dasgd_delay_guideline(double t_c, double t_p, int32_t *d, int32_t *tau);
+
+/* The guideline applied to this context's own measurements.  Requires DASGD_FLAG_TIMING and at least
+ * one timed local step and one timed mean.  t_c = average device time of the mean kernel; t_p = average
+ * device time of the local-step kernel + extra_tp_ms (the caller's forward/backward time per step,
+ * 0 if the gradients are precomputed).  Synchronises.  Outputs: *d, *tau, and (if non-NULL) the two
+ * times in milliseconds. */
+dasgd_status dasgd_advise_delay(dasgd_ctx *ctx, double extra_tp_ms, int32_t *d, int32_t *tau, double *t_c_ms,
+                                double *t_p_ms);
+
 /* Number of kernels this context has launched so far. */
 dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches);
 

@@ -59,6 +59,9 @@ def bind(path: str) -> ctypes.CDLL:
     L.oracle_dasgd_merge.argtypes = [vp]
     L.oracle_dasgd_step.argtypes = [vp, vp, f32]
     L.oracle_dasgd_threads.argtypes = []
+    f64, pi32 = ctypes.c_double, ctypes.POINTER(i32)
+    L.oracle_dasgd_delay_guideline.argtypes = [f64, f64, pi32, pi32]
+    L.oracle_dasgd_delay_from_system.argtypes = [f64, f64, f64, f64, f64, f64, pi32, pi32]
     return L
 
 
@@ -71,6 +74,21 @@ def _lib(omp: bool) -> ctypes.CDLL:
 
 class OracleError(RuntimeError):
     pass
+
+
+def delay_guideline(t_c: float, t_p: float):
+    """(d, tau) of the paper's guideline: smallest d with t_c < d*t_p; tau = d + 1."""
+    d, tau = ctypes.c_int32(), ctypes.c_int32()
+    if _lib(False).oracle_dasgd_delay_guideline(t_c, t_p, ctypes.byref(d), ctypes.byref(tau)) != 0:
+        raise OracleError("delay_guideline: need t_c >= 0 and t_p > 0")
+    return d.value, tau.value
+
+
+def delay_from_system(m, n_p, BW, B_l, FLOP, FLOPS):
+    d, tau = ctypes.c_int32(), ctypes.c_int32()
+    if _lib(False).oracle_dasgd_delay_from_system(m, n_p, BW, B_l, FLOP, FLOPS, ctypes.byref(d), ctypes.byref(tau)) != 0:
+        raise OracleError("delay_from_system: bad arguments")
+    return d.value, tau.value
 
 
 def _ptr(a):

@@ -216,6 +216,22 @@ int oracle_dasgd_step(oracle_dasgd *o, const void *g, float lr) {
   return rc;
 }
 
+// Eq. 3: d > t_c / t_p, smallest such positive integer; Section VI-D: tau = d + 1.
+int oracle_dasgd_delay_guideline(double t_c, double t_p, int32_t *d, int32_t *tau) {
+  if (!(t_c >= 0.0) || !(t_p > 0.0) || !d || !tau) return ORACLE_ERR_ARG;
+  int32_t k = 1;
+  while (!(t_c < static_cast<double>(k) * t_p)) ++k;
+  *d = k;
+  *tau = k + 1;
+  return ORACLE_OK;
+}
+
+int oracle_dasgd_delay_from_system(double m, double n_p, double BW, double B_l, double FLOP, double FLOPS,
+                                   int32_t *d, int32_t *tau) {
+  if (!(BW > 0.0) || !(FLOPS > 0.0)) return ORACLE_ERR_ARG;
+  return oracle_dasgd_delay_guideline(m * n_p / BW, B_l * FLOP / FLOPS, d, tau);
+}
+
 int oracle_dasgd_threads(void) {
 #ifdef _OPENMP
   return omp_get_max_threads();

@@ -31,8 +31,8 @@
  * the minibatch-SGD and Local-SGD special cases (Eq. 1, Section II-C-3), the
  * averaged-model recursion of Section III-C-1, the deviation contraction used in
  * the proof of the theorem (Appendix), closed forms for momentum and weight
- * decay, torch.optim.SGD for the momentum/weight-decay local step, and torch's
- * bfloat16 cast for the rounding.
+ * decay, torch.optim.SGD for the momentum/weight-decay local step, torch's
+ * bfloat16 cast for the rounding, and the paper's Table II for the delay guideline.
  * Parity unpinned by the paper: schedules with d > tau (the paper assumes
  * d <= tau) -- defined here by pipelining snapshots, checked by invariants only.
  */
@@ -74,6 +74,14 @@ int oracle_dasgd_merge(oracle_dasgd *o);   /* blend the OLDEST pending mean, the
 
 /* One iteration of the schedule: local step; merge if one lands; snapshot+mean if due. */
 int oracle_dasgd_step(oracle_dasgd *o, const void *g, float lr);
+
+/* Delay guideline (Section III-D, Eq. 3; Section VI-C and VI-D): the averaging is hidden when
+ * t_c < d * t_p, so d is the smallest positive integer with that property, and tau = d + 1.
+ * Pinned against every row of the paper's Table II.  Returns ORACLE_ERR_ARG unless t_c >= 0, t_p > 0. */
+int oracle_dasgd_delay_guideline(double t_c, double t_p, int32_t *d, int32_t *tau);
+/* The same from system parameters (Eq. 3): t_c = m*n_p/BW, t_p = B_l*FLOP/FLOPS. */
+int oracle_dasgd_delay_from_system(double m, double n_p, double BW, double B_l, double FLOP, double FLOPS,
+                                   int32_t *d, int32_t *tau);
 
 int oracle_dasgd_threads(void); /* OpenMP threads the element loops use (1 if built without) */
 

@@ -29,7 +29,7 @@ EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
     "dasgd_step", "dasgd_step_host", "dasgd_get_weights", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
-    "dasgd_average_merge_noalloc",
+    "dasgd_average_merge_noalloc", "dasgd_delay_guideline", "dasgd_advise_delay",
 ]
 
 
@@ -80,6 +80,9 @@ def _load() -> ctypes.CDLL:
     L.dasgd_last_error.restype = ctypes.c_char_p
     L.dasgd_destroy.argtypes = [vp]
     L.dasgd_average_merge_noalloc.argtypes = [vp, i32, i64, i64, f32, i32, vp, ctypes.c_char_p, i64]
+    f64, pi32, pf64 = ctypes.c_double, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)
+    L.dasgd_delay_guideline.argtypes = [f64, f64, pi32, pi32]
+    L.dasgd_advise_delay.argtypes = [vp, f64, pi32, pi32, pf64, pf64]
     L.dasgd_version.argtypes = []
     L.dasgd_version.restype = ctypes.c_char_p
     return L
@@ -166,6 +169,23 @@ def dasgd_get_kernel_timing(ctx, which: int):
 
 def dasgd_reset_timing(ctx):
     _check(_L.dasgd_reset_timing(ctx), ctx)
+
+
+def dasgd_delay_guideline(t_c: float, t_p: float):
+    """(d, tau): smallest d with t_c < d*t_p, tau = d + 1 (the paper's guideline, Eq. 3)."""
+    d, tau = ctypes.c_int32(), ctypes.c_int32()
+    st = _L.dasgd_delay_guideline(t_c, t_p, ctypes.byref(d), ctypes.byref(tau))
+    if st != DASGD_OK:
+        raise DasgdError(st, "delay_guideline: need t_c >= 0 and t_p > 0")
+    return d.value, tau.value
+
+
+def dasgd_advise_delay(ctx, extra_tp_ms: float = 0.0):
+    """(d, tau, t_c_ms, t_p_ms) from the context's own timings (needs DASGD_FLAG_TIMING)."""
+    d, tau, tc, tp = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_double(), ctypes.c_double()
+    _check(_L.dasgd_advise_delay(ctx, extra_tp_ms, ctypes.byref(d), ctypes.byref(tau), ctypes.byref(tc),
+                                 ctypes.byref(tp)), ctx)
+    return d.value, tau.value, tc.value, tp.value
 
 
 def dasgd_get_launches(ctx) -> int:
@@ -328,6 +348,9 @@ class DaSGD:
 
     def reset_timing(self):
         dasgd_reset_timing(self.ctx)
+
+    def advise_delay(self, extra_tp_ms=0.0):
+        return dasgd_advise_delay(self.ctx, extra_tp_ms)
 
     @property
     def launches(self):

@@ -772,6 +772,40 @@ dasgd_status dasgd_reset_timing(dasgd_ctx *ctx) {
   return DASGD_OK;
 }
 
+dasgd_status dasgd_delay_guideline(double t_c, double t_p, int32_t *d, int32_t *tau) {
+  if (!d || !tau || !(t_c >= 0.0) || !(t_p > 0.0)) return DASGD_ERR_INVALID_ARG;
+  // d > t_c / t_p (Eq. 3): step up from the quotient so that rounding in the division cannot
+  // produce a d that violates t_c < d * t_p or is larger than necessary
+  double q = t_c / t_p;
+  if (q > 1e9) return DASGD_ERR_INVALID_ARG;
+  int64_t k = (int64_t)q;  // floor, q >= 0
+  if (k < 1) k = 1;
+  while (k > 1 && t_c < (double)(k - 1) * t_p) --k;
+  while (!(t_c < (double)k * t_p)) ++k;
+  *d = (int32_t)k;
+  *tau = (int32_t)k + 1;
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_advise_delay(dasgd_ctx *ctx, double extra_tp_ms, int32_t *d, int32_t *tau, double *t_c_ms,
+                                double *t_p_ms) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!d || !tau || !(extra_tp_ms >= 0.0)) return fail(ctx, DASGD_ERR_INVALID_ARG, "advise_delay: bad arguments");
+  if (!(ctx->cfg.flags & DASGD_FLAG_TIMING)) return fail(ctx, DASGD_ERR_BAD_STATE, "advise_delay: DASGD_FLAG_TIMING not set");
+  dasgd_status st = dasgd_sync(ctx);
+  if (st != DASGD_OK) return st;
+  DeviceGuard guard(ctx->cfg.device);
+  harvest(ctx, true);
+  if (ctx->span_n[TAG_STEP] < 1 || ctx->span_n[TAG_MEAN] < 1)
+    return fail(ctx, DASGD_ERR_BAD_STATE, "advise_delay: needs at least one timed local step and one timed mean");
+  const double tc = ctx->span_ms[TAG_MEAN] / (double)ctx->span_n[TAG_MEAN];
+  const double tp = ctx->span_ms[TAG_STEP] / (double)ctx->span_n[TAG_STEP] + extra_tp_ms;
+  if (t_c_ms) *t_c_ms = tc;
+  if (t_p_ms) *t_p_ms = tp;
+  if (dasgd_delay_guideline(tc, tp, d, tau) != DASGD_OK) return fail(ctx, DASGD_ERR_INVALID_ARG, "advise_delay: degenerate timings");
+  return DASGD_OK;
+}
+
 dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches) {
   if (!ctx || !launches) return DASGD_ERR_INVALID_ARG;
   *launches = ctx->launches;

@@ -8,6 +8,7 @@ import pytest
 
 import oracle
 from tests import test_oracle_golden as G
+from tests import test_delay_guideline as D
 from tests import test_oracle_invariants as I
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "dasgd_oracle.cpp")
@@ -29,6 +30,9 @@ MUTATIONS = {
     "delta merge sign": ("wi + (avg - static_cast<double>(q.snap[i]))", "wi - (avg - static_cast<double>(q.snap[i]))"),
     "delta merge uses the current weights as the snapshot": ("static_cast<double>(q.snap[i])))", "wi))"),
     "merge takes the newest mean": ("const Pending &q = o->pending.front();", "const Pending &q = o->pending.back();"),
+    "guideline: tau equals d": ("*tau = k + 1;", "*tau = k;"),
+    "guideline: non-strict inequality": ("while (!(t_c < static_cast<double>(k) * t_p)) ++k;",
+                                         "while (!(t_c <= static_cast<double>(k) * t_p)) ++k;"),
     "momentum merged too": ("o->pending.pop_front();\n  return ORACLE_OK;", "for (auto &x : o->m) x *= o->xi;\n  o->pending.pop_front();\n  return ORACLE_OK;"),
 }
 
@@ -52,6 +56,10 @@ def battery():
     I.test_weight_decay_closed_form_zero_gradient()
     I.test_bf16_rounding_matches_torch_cast()
     I.test_bf16_mode_master_equals_f32_run_on_widened_gradients()
+    for row in D.table2():
+        D.test_oracle_reproduces_table2(row)
+    assert oracle.delay_guideline(1.0, 1.0) == (2, 3)      # Eq. 3 is strict: d > t_c / t_p
+    assert oracle.delay_guideline(0.0, 1.0) == (1, 2)      # a delay of at least one step
 
 
 def build_variant(tmp_path, text, tag):
@@ -83,7 +91,7 @@ def test_planted_mistake_is_caught(name, tmp_path, swap_lib):
     if MUTATIONS[name] is None:
         a = text.index("  if (d > 0 && u - d >= tau && (u - d) % tau == 0) {")
         b = text.index("  if (u % tau == 0) {")
-        c = text.index("  return rc;\n}\n\nint oracle_dasgd_threads")
+        c = text.index("  return rc;\n}\n", b)
         merge_block, snap_block = text[a:b], text[b:c]
         mutated = text[:a] + snap_block + merge_block + text[c:]
     else:
