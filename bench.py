@@ -211,25 +211,6 @@ def whole_job(ms_local: float, units_per_rank: float, dist=None, device="cpu"):
     return ms, world * units_per_rank / (ms * 1e-3)
 
 
-def event_gap_ms(n=50):
-    """Median device time between two CUDA events that bracket a wait on an already-completed event."""
-    st = torch.cuda.Stream()
-    done = torch.cuda.Event()
-    with torch.cuda.stream(st):
-        done.record()
-    st.synchronize()
-    pairs = []
-    for _ in range(n):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(st):
-            a.record()
-            st.wait_event(done)
-            b.record()
-        pairs.append((a, b))
-    st.synchronize()
-    return statistics.median(a.elapsed_time(b) for a, b in pairs)
-
-
 def run_ours(args, wl, name):
     from paper_2006_00441_b200 import binding as B
 
@@ -331,15 +312,28 @@ def run_ours(args, wl, name):
         if n_k:
             gbs = nbytes / 1e9 / (ms_k / n_k * 1e-3)
             alone[kname] = {"ms": ms_k / n_k, "GB/s": gbs, "frac": gbs / peak}
-    # Hidden fraction of the averaging.  "raw": every microsecond between the two events that bracket
-    # the main stream's wait counts as stall, including the cost of the events themselves; "net": the
-    # same minus that cost, measured as the gap between two events around a wait that is already
-    # satisfied on an otherwise idle stream.
-    hidden = hidden_net = gap_ms = None
+    # Hidden fraction of the averaging: every microsecond between the two events that bracket the main
+    # stream's wait for a mean counts as stall (that includes the cost of the two events themselves).
+    hidden = None
     if kt["mean"][0] and kt["mean"][1] > 0:
         hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
-        gap_ms = event_gap_ms()
-        hidden_net = min(1.0, max(0.0, 1.0 - max(0.0, kt["stall"][1] - kt["stall"][0] * gap_ms) / kt["mean"][1]))
+
+    # ---- ablation: the same work with the mean computed inside the step kernel (no side stream)
+    ablation = None
+    if not args.no_ablation:
+        eng = B.DaSGD(K, P, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"],
+                      flags=B.DASGD_FLAG_INLINE_MEAN, dtype=B.DASGD_BF16_MASTER_F32 if bf16 else B.DASGD_F32,
+                      device=local_rank, order_after_current=False, snapshot_arrays=False)
+        eng.set_state(inputs.shared_start(seed, P, wl["w_std"], device="cuda"))
+        ms_a, launches_a = timed_loop(eng, args.steps, args.warmup, dev_step)
+        bytes_a = (step_bytes(wl) * wl["tau"] + 8.0 / K) / wl["tau"]
+        ablation = {"schedule": "inline mean: one kernel per iteration, mean summed in registers, no snapshot, "
+                                "no side stream (same results; the averaging is no longer asynchronous)",
+                    "value": world * K * P * args.steps / (ms_a * 1e-3), "unit": UNIT, "ms_per_step": ms_a / args.steps,
+                    "gpu_launches": launches_a, "bytes_per_update": bytes_a,
+                    "whole_path_gbs": K * P * args.steps / (ms_a * 1e-3) * bytes_a / 1e9}
+        eng.close()
+        del eng
 
     # ---- end to end: gradients start in page-locked host memory every step
     e2e = None
@@ -393,9 +387,9 @@ def run_ours(args, wl, name):
                      "traffic": None,
                      "alone": alone},
         "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
-        "averaging_hidden_frac": hidden, "averaging_hidden_frac_net_of_event_cost": hidden_net,
-        "event_pair_gap_ms": gap_ms,
+        "averaging_hidden_frac": hidden,
         "whole_path_gbs": value / world * path_bytes_per_update(wl) / 1e9,
+        "ablation_inline_mean": ablation,
         "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
     }
     return line
@@ -412,6 +406,9 @@ def run_sweep(args):
                 if line:
                     keep = {k: line[k] for k in ("value", "ms_per_step", "gpu_launches", "averaging_hidden_frac",
                                                  "whole_path_gbs", "kernels_ms_per_launch")}
+                    if line.get("ablation_inline_mean"):
+                        keep["inline_mean_value"] = line["ablation_inline_mean"]["value"]
+                        keep["inline_mean_gbs"] = line["ablation_inline_mean"]["whole_path_gbs"]
                     keep.update(K=K, tau=tau, d=d, local_step_alone_gbs=line["roofline"]["alone"]["local_step"]["GB/s"])
                     print(json.dumps(keep), flush=True)
 
@@ -441,6 +438,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-fuse", action="store_true", help="run the unfused schedule (separate snapshot copy and merge)")
+    ap.add_argument("--no-ablation", action="store_true", help="skip the inline-mean ablation leg")
     ap.add_argument("--sweep", action="store_true", help="run the K x tau x d sweep instead (one JSON line per point)")
     args = ap.parse_args()
     if args.warmup < 3:

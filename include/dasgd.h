@@ -71,6 +71,14 @@ typedef enum {
                                          between arrays: ask dasgd_get_weights where they are.  Results are
                                          the same as without the flag.  FUSE_SNAPSHOT has no effect.        */
 
+#define DASGD_FLAG_INLINE_MEAN 0x10u   /* dasgd_step runs ONE kernel per iteration: each thread walks the K rows
+                                         of its parameters, does the local step and the merge that lands, and,
+                                         when a snapshot is due, writes the mean of the K results directly.  No
+                                         snapshot array is read or written (cfg.snap may be NULL) and the side
+                                         stream stays idle: fastest schedule on one GPU, same results, but the
+                                         mean is no longer computed asynchronously.  xi-blend merge only.  The
+                                         explicit snapshot/average/merge calls keep working if snap is given. */
+
 typedef struct dasgd_config {
   int32_t K;            /* workers (the paper's M), >= 1                                              */
   int32_t tau;          /* local steps between snapshots, >= 1                                        */

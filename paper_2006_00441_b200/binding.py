@@ -24,6 +24,7 @@ DASGD_ERR_CUDA, DASGD_ERR_TIMEOUT, DASGD_ERR_UNSUPPORTED = 4, 5, 6
 DASGD_F32, DASGD_BF16_MASTER_F32 = 0, 1
 DASGD_MERGE_XI, DASGD_MERGE_DELTA = 0, 1
 DASGD_FLAG_TIMING, DASGD_FLAG_FUSE_SNAPSHOT, DASGD_FLAG_FUSE_MERGE, DASGD_FLAG_ROTATE_SNAPSHOT = 0x1, 0x2, 0x4, 0x8
+DASGD_FLAG_INLINE_MEAN = 0x10
 
 EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
@@ -226,7 +227,7 @@ class DaSGD:
 
     def __init__(self, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=DASGD_F32,
                  merge_mode=DASGD_MERGE_XI, flags=0, n_slots=None, ld=None, device=0, host_staging=False,
-                 sync_timeout_ms=0, order_after_current=True):
+                 sync_timeout_ms=0, order_after_current=True, snapshot_arrays=True):
         if not torch.cuda.is_available():
             raise RuntimeError("DaSGD needs a CUDA device; there is no CPU implementation")
         self.K, self.P, self.tau, self.d = K, P, tau, d
@@ -242,7 +243,9 @@ class DaSGD:
         self._w0 = torch.zeros((K, self.ld), dtype=torch.float32, device=dev)
         self.m = torch.zeros((K, self.ld), dtype=torch.float32, device=dev) if momentum != 0.0 else None
         self.w_lp = torch.zeros((K, self.ld), dtype=torch.bfloat16, device=dev) if dtype == DASGD_BF16_MASTER_F32 else None
-        self.snap = torch.empty((self.n_slots, K, self.ld), dtype=torch.float32, device=dev)
+        # the inline-mean schedule never touches snapshot arrays; they can be left out to save memory
+        self.snap = (torch.empty((self.n_slots, K, self.ld), dtype=torch.float32, device=dev)
+                     if snapshot_arrays or not (flags & DASGD_FLAG_INLINE_MEAN) else None)
         self.mean = torch.empty((self.n_slots, self.ld), dtype=torch.float32, device=dev)
         n_stage = int(host_staging) if host_staging in (0, 1, 2, True, False) else 0
         self.g_stage = torch.empty((n_stage, K, self.ld), dtype=self.gdtype, device=dev) if n_stage else None
@@ -259,7 +262,8 @@ class DaSGD:
         cfg.w = self._w0.data_ptr()
         cfg.m = self.m.data_ptr() if self.m is not None else None
         cfg.w_lp = self.w_lp.data_ptr() if self.w_lp is not None else None
-        cfg.snap, cfg.mean = self.snap.data_ptr(), self.mean.data_ptr()
+        cfg.snap = self.snap.data_ptr() if self.snap is not None else None
+        cfg.mean = self.mean.data_ptr()
         cfg.g_stage = self.g_stage.data_ptr() if self.g_stage is not None else None
         cfg.n_stage = n_stage
         cfg.main_stream, cfg.side_stream = self.main.cuda_stream, self.side.cuda_stream

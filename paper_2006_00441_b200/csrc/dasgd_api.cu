@@ -298,6 +298,44 @@ dasgd_status launch_merge(dasgd_ctx *c, const Params &p, bool snap) {
   return snap ? launch_merge_t<false, 1, true>(c, p) : launch_merge_t<false, 1, false>(c, p);
 }
 
+template <bool BF16, bool MOM, bool MERGE, bool MEANOUT>
+dasgd_status launch_allk_t(dasgd_ctx *c, const Params &p, bool vec) {
+  constexpr int EPU = BF16 ? 8 : 4;
+  long long done = 0;
+  if (vec) {
+    const long long units = p.P / EPU;
+    if (units > 0) {
+      dasgd::k_step_allk_vec<BF16, MOM, MERGE, MEANOUT><<<blocks_for(units, kThreads), kThreads, 0, c->s0>>>(p);
+      c->launches++;
+    }
+    done = units * EPU;
+  }
+  if (done < p.P) {
+    dasgd::k_step_allk_scalar<BF16, MOM, MERGE, MEANOUT>
+        <<<blocks_for(p.P - done, kThreads), kThreads, 0, c->s0>>>(p, done);
+    c->launches++;
+  }
+  CU(c, cudaGetLastError());
+  return DASGD_OK;
+}
+
+template <bool BF16, bool MOM>
+dasgd_status launch_allk_m(dasgd_ctx *c, const Params &p, bool vec, bool merge, bool meanout) {
+  if (merge) return meanout ? launch_allk_t<BF16, MOM, true, true>(c, p, vec) : launch_allk_t<BF16, MOM, true, false>(c, p, vec);
+  return meanout ? launch_allk_t<BF16, MOM, false, true>(c, p, vec) : launch_allk_t<BF16, MOM, false, false>(c, p, vec);
+}
+
+dasgd_status launch_allk(dasgd_ctx *c, const Params &p, bool vec, bool merge, bool meanout) {
+  const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32;
+  const bool mom = c->cfg.momentum != 0.0f;
+  const int sp = span_begin(c, TAG_STEP, c->s0);
+  dasgd_status st;
+  if (bf16) st = mom ? launch_allk_m<true, true>(c, p, vec, merge, meanout) : launch_allk_m<true, false>(c, p, vec, merge, meanout);
+  else st = mom ? launch_allk_m<false, true>(c, p, vec, merge, meanout) : launch_allk_m<false, false>(c, p, vec, merge, meanout);
+  span_end(c, sp, c->s0);
+  return st;
+}
+
 // -------------------------------------------------------------- slot operations
 
 int find_free_slot(const dasgd_ctx *c) {
@@ -426,7 +464,11 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   const int need = c.d == 0 ? 1 : (c.d + c.tau - 1) / c.tau;
   if (c.n_slots < need)
     return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: n_slots must be >= max(1, ceil(d/tau))");
-  if (!c.w || !c.snap || !c.mean) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: w, snap and mean must not be NULL");
+  const bool inline_mean = (c.flags & DASGD_FLAG_INLINE_MEAN) != 0;
+  if (inline_mean && c.merge_mode != DASGD_MERGE_XI)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: DASGD_FLAG_INLINE_MEAN supports the xi-blend merge only");
+  if (!c.w || !c.mean || (!c.snap && !inline_mean))
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: w, snap and mean must not be NULL");
   if (c.momentum != 0.0f && !c.m) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: momentum != 0 needs m");
   if (c.dtype == DASGD_BF16_MASTER_F32 && !c.w_lp)
     return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: bf16 mode needs w_lp");
@@ -454,7 +496,7 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   ctx->vec = (c.ld % ctx->epu) == 0;
   ctx->rotate = (c.flags & DASGD_FLAG_ROTATE_SNAPSHOT) != 0;
   ctx->pool.push_back(static_cast<float *>(c.w));
-  for (int i = 0; i < c.n_slots; ++i)
+  for (int i = 0; c.snap && i < c.n_slots; ++i)
     ctx->pool.push_back(static_cast<float *>(c.snap) + (size_t)i * c.K * c.ld);
   ctx->frozen.assign(ctx->pool.size(), -1);
   DeviceGuard guard(c.device);
@@ -558,6 +600,7 @@ dasgd_status op_merge(dasgd_ctx *c, int slot, int snap_buf) {
 dasgd_status op_snapshot(dasgd_ctx *c, int already_in) {
   const int slot = find_free_slot(c);
   if (slot < 0) return fail(c, DASGD_ERR_NO_SLOT, "snapshot: every slot holds a pending average");
+  if (c->pool.size() < 2) return fail(c, DASGD_ERR_BAD_STATE, "snapshot: no snapshot arrays were configured (cfg.snap)");
   if (c->rotate) return mark_snapped(c, slot, c->cur);
   int buf = already_in;
   if (buf < 0) {
@@ -569,6 +612,51 @@ dasgd_status op_snapshot(dasgd_ctx *c, int already_in) {
     if (st != DASGD_OK) return st;
   }
   return mark_snapped(c, slot, buf);
+}
+
+// One iteration of the inline-mean schedule: everything on the main stream, one kernel (two when
+// d == 0, because the blend then needs the mean of the very weights this kernel produces).
+dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, bool s_due) {
+  if (c->frozen[c->cur] >= 0)
+    return fail(c, DASGD_ERR_BAD_STATE, "step: a snapshot taken with dasgd_snapshot is pending; merge it first");
+  Params p = base_params(c);
+  p.g = grads;
+  p.lr = lr;
+  if (m_due) {
+    if (c->pending.empty()) return fail(c, DASGD_ERR_BAD_STATE, "step: no mean is pending");
+    const int ms = c->pending.front();
+    if (c->slots[ms].state != SLOT_AVERAGING)
+      return fail(c, DASGD_ERR_BAD_STATE, "step: the oldest snapshot has no mean yet");
+    if (c->slots[ms].buf >= 0) {  // it came from dasgd_snapshot/dasgd_average_async: order after the side stream
+      CU(c, cudaStreamWaitEvent(c->s0, c->slots[ms].e_avg, 0));
+    }
+    p.mean = mean_ptr(c, ms);
+    release_oldest(c);  // its mean is read by this iteration's kernel; the slot may be refilled by it
+  }
+  int slot = -1;
+  if (s_due) {
+    slot = find_free_slot(c);
+    if (slot < 0) return fail(c, DASGD_ERR_NO_SLOT, "step: no free slot for the mean");
+    p.mean_out = mean_ptr(c, slot);
+  }
+  dasgd_status st = launch_allk(c, p, grads_vec_ok(c, grads), m_due, s_due);
+  if (st != DASGD_OK) return st;
+  c->t += 1;
+  if (s_due) {
+    Slot &sl = c->slots[slot];
+    sl.state = SLOT_AVERAGING;  // the mean is already on its way, on this same stream
+    sl.s = c->t;
+    sl.buf = -1;                // no snapshot array belongs to it
+    c->pending.push_back(slot);
+    if (c->cfg.d == 0) {        // Local SGD: blend it back at once
+      Params q = base_params(c);
+      q.mean = mean_ptr(c, slot);
+      st = launch_merge(c, q, false);
+      if (st != DASGD_OK) return st;
+      release_oldest(c);
+    }
+  }
+  return DASGD_OK;
 }
 
 }  // namespace
@@ -612,6 +700,7 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
   const int64_t u = ctx->t + 1;
   const bool m_due = merge_due(ctx, u);
   const bool s_due = (u % cfg.tau) == 0;
+  if (cfg.flags & DASGD_FLAG_INLINE_MEAN) return step_inline(ctx, grads, lr, m_due, s_due);
   const bool fuse_merge = m_due && (cfg.flags & DASGD_FLAG_FUSE_MERGE) && cfg.d >= 2;
   // copy mode only: let the kernel that last writes w in this iteration also store the snapshot
   const bool fuse_snap = s_due && !ctx->rotate && (cfg.flags & DASGD_FLAG_FUSE_SNAPSHOT);

@@ -390,4 +390,123 @@ __global__ void __launch_bounds__(kThreads) k_merge_scalar(const Params p, long 
   }
 }
 
+// ---------------------------------------------------------------- whole iteration in one kernel
+// "Inline mean" schedule: one thread owns one unit of the parameter axis and walks the K rows doing
+// the local step; if a merge lands on this iteration it blends with the stored mean (kept in
+// registers); if a snapshot is due it sums the resulting weights of the K rows and writes their mean.
+// The mean therefore needs no snapshot array and no second pass over HBM.  Same arithmetic and the
+// same summation tree as the separate kernels, so the results are bit-identical to theirs.
+// mean (read) and mean_out (written) may be the same array: a thread reads its elements of the old
+// mean before it writes the new ones.
+
+template <bool BF16, bool MOM, bool MERGE, bool MEANOUT>
+__global__ void __launch_bounds__(kThreads) k_step_allk_vec(const Params p) {
+  constexpr int EPU = BF16 ? 8 : 4;
+  constexpr int F4 = EPU / 4;
+  constexpr int KB = BF16 ? 2 : 4;  // rows loaded together; rows are taken in groups of 4
+  const long long u = (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (u >= p.P / EPU) return;
+  const long long e = u * EPU;
+  float4 a[F4], acc[F4][4];
+#pragma unroll
+  for (int f = 0; f < F4; ++f) {
+    if (MERGE) a[f] = __ldg(reinterpret_cast<const float4 *>(p.mean + e) + f);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[f][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int k0 = 0; k0 < p.K; k0 += 4) {
+#pragma unroll
+    for (int h = 0; h < 4; h += KB) {
+      float4 w[KB][F4], m[KB][F4], g[KB][F4];
+#pragma unroll
+      for (int j = 0; j < KB; ++j) {
+        const int k = k0 + h + j;
+        if (k >= p.K) continue;
+        const long long off = (long long)k * p.ld + e;
+        if (BF16) {
+          const uint4 gb = ld_stream(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.g) + off));
+          g[j][0] = make_float4(bf16_bits_to_f32(gb.x & 0xFFFFu), bf16_bits_to_f32(gb.x >> 16),
+                                bf16_bits_to_f32(gb.y & 0xFFFFu), bf16_bits_to_f32(gb.y >> 16));
+          g[j][F4 - 1] = make_float4(bf16_bits_to_f32(gb.z & 0xFFFFu), bf16_bits_to_f32(gb.z >> 16),
+                                     bf16_bits_to_f32(gb.w & 0xFFFFu), bf16_bits_to_f32(gb.w >> 16));
+        } else {
+          g[j][0] = ld_stream(reinterpret_cast<const float4 *>(static_cast<const float *>(p.g) + off));
+        }
+#pragma unroll
+        for (int f = 0; f < F4; ++f) {
+          w[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.w + off) + f);
+          if (MOM) m[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.m + off) + f);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < KB; ++j) {
+        const int k = k0 + h + j;
+        if (k >= p.K) continue;
+        const long long off = (long long)k * p.ld + e;
+#pragma unroll
+        for (int f = 0; f < F4; ++f) {
+          float4 x = w[j][f];
+          float4 y = MOM ? m[j][f] : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 gg = g[j][f];
+          step_elem<MOM>(x.x, y.x, gg.x, p);
+          step_elem<MOM>(x.y, y.y, gg.y, p);
+          step_elem<MOM>(x.z, y.z, gg.z, p);
+          step_elem<MOM>(x.w, y.w, gg.w, p);
+          if (MERGE) {
+            DASGD_F4_APPLY(x, blend_xi(x.x, a[f].x, p), blend_xi(x.y, a[f].y, p), blend_xi(x.z, a[f].z, p),
+                           blend_xi(x.w, a[f].w, p))
+          }
+          st_stream(reinterpret_cast<float4 *>(p.w_out + off) + f, x);
+          if (MOM) st_stream(reinterpret_cast<float4 *>(p.m + off) + f, y);
+          if (MEANOUT) add4(acc[f][h + j], x);   // (k mod 4) == h + j because k0 is a multiple of 4
+          w[j][f] = x;
+        }
+        if (BF16) {
+          uint4 o;
+          o.x = pack_bf16x2(w[j][0].x, w[j][0].y);
+          o.y = pack_bf16x2(w[j][0].z, w[j][0].w);
+          o.z = pack_bf16x2(w[j][F4 - 1].x, w[j][F4 - 1].y);
+          o.w = pack_bf16x2(w[j][F4 - 1].z, w[j][F4 - 1].w);
+          st_stream(reinterpret_cast<uint4 *>(p.w_lp + off), o);
+        }
+      }
+    }
+  }
+  if (MEANOUT) {
+    const float kf = (float)p.K;
+#pragma unroll
+    for (int f = 0; f < F4; ++f) {
+      add4(acc[f][0], acc[f][1]);
+      add4(acc[f][2], acc[f][3]);
+      add4(acc[f][0], acc[f][2]);
+      float4 r;
+      r.x = __fdiv_rn(acc[f][0].x, kf); r.y = __fdiv_rn(acc[f][0].y, kf);
+      r.z = __fdiv_rn(acc[f][0].z, kf); r.w = __fdiv_rn(acc[f][0].w, kf);
+      reinterpret_cast<float4 *>(p.mean_out + e)[f] = r;
+    }
+  }
+}
+
+template <bool BF16, bool MOM, bool MERGE, bool MEANOUT>
+__global__ void __launch_bounds__(kThreads) k_step_allk_scalar(const Params p, long long p0) {
+  const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (col >= p.P) return;
+  const float a = MERGE ? p.mean[col] : 0.0f;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int k = 0; k < p.K; ++k) {
+    const long long i = (long long)k * p.ld + col;
+    float w = p.w[i], m = MOM ? p.m[i] : 0.0f;
+    const float g = BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(p.g)[i])
+                         : static_cast<const float *>(p.g)[i];
+    step_elem<MOM>(w, m, g, p);
+    if (MERGE) w = blend_xi(w, a, p);
+    p.w_out[i] = w;
+    if (MOM) p.m[i] = m;
+    if (BF16) p.w_lp[i] = __float2bfloat16_rn(w);
+    if (MEANOUT) acc[k & 3] = __fadd_rn(acc[k & 3], w);
+  }
+  if (MEANOUT)
+    p.mean_out[col] = __fdiv_rn(__fadd_rn(__fadd_rn(acc[0], acc[1]), __fadd_rn(acc[2], acc[3])), (float)p.K);
+}
+
 }  // namespace dasgd

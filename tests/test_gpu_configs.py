@@ -119,11 +119,27 @@ def test_config2_resnet50_sized_200_steps(B):
                 checkpoints=(1, 2, 100))
 
 
+def test_config2_inline_mean_schedule(B):
+    run_sampled(B, K=8, P=25_600_000, tau=1, d=1, xi=0.25, mom=0.9, wd=1e-4, lr=0.1, T=100, g_std=1e-3 ** 0.5,
+                flags=0x10)
+
+
+@pytest.mark.parametrize("K,tau,d", [(32, 1, 2), (2, 4, 1), (16, 2, 2)])
+def test_config4_points_inline_mean_schedule(B, K, tau, d):
+    run_sampled(B, K=K, P=25_600_000, tau=tau, d=d, xi=0.25, mom=0.9, wd=0.0, lr=0.1, T=100, g_std=1e-3 ** 0.5,
+                ring=2, seed=K + tau + d, flags=0x10)
+
+
 # ---------------------------------------------------------------- config 3: BERT-large-sized, bf16
 
 def test_config3_bert_large_sized_bf16_50_steps(B):
     run_sampled(B, K=4, P=335_000_000, tau=2, d=1, xi=0.25, mom=0.9, wd=0.0, lr=1e-3, T=50, g_std=1e-2,
                 dtype=1, ring=2, checkpoints=(1, 3, 25))
+
+
+def test_config3_inline_mean_schedule(B):
+    run_sampled(B, K=4, P=335_000_000, tau=2, d=1, xi=0.25, mom=0.9, wd=0.0, lr=1e-3, T=50, g_std=1e-2,
+                dtype=1, ring=2, flags=0x10)
 
 
 # ---------------------------------------------------------------- config 4: the sweep

@@ -13,7 +13,7 @@ from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, make_pair,
 
 pytestmark = pytest.mark.gpu
 
-FUSE_SNAP, FUSE_MERGE, ROTATE = 0x2, 0x4, 0x8
+FUSE_SNAP, FUSE_MERGE, ROTATE, INLINE = 0x2, 0x4, 0x8, 0x10
 # f32 vector tile = 256 threads * 4 units * 4 elements = 4096 elements; bf16 tile = 256*2*8 = 4096
 SIZES = [1, 3, 4, 7, 8, 1000, 4096, 3 * 4096 + 1029]
 
@@ -91,9 +91,11 @@ SCHEDULES = [(1, 1), (2, 1), (4, 1), (1, 2), (2, 2), (4, 2), (2, 3), (3, 0), (1,
 
 
 @pytest.mark.parametrize("tau,d", SCHEDULES)
-@pytest.mark.parametrize("flags", [0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE])
+@pytest.mark.parametrize("flags", [0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE, INLINE])
 @pytest.mark.parametrize("K,dtype,mode", [(4, 0, 0), (3, 1, 0), (8, 0, 1)])
 def test_free_running_100_steps(B, tau, d, flags, K, dtype, mode):
+    if flags & INLINE and mode == 1:
+        pytest.skip("the inline-mean schedule has no delta merge")
     P, T = 2 * 4096 + 77, 100
     ld = (P + 7) // 8 * 8
     w0 = inputs.shared_start(2, P, 0.02).numpy()
@@ -123,7 +125,7 @@ def test_fused_schedules_are_bit_identical_to_unfused(B, tau, d, dtype, mode):
     w0 = inputs.shared_start(4, P, 0.02)
     gd = torch.bfloat16 if dtype else torch.float32
     outs = []
-    for flags in (0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE):
+    for flags in (0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE) + ((INLINE,) if mode == 0 else ()):
         gpu = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld)
         gpu.set_state(w0)
         for t in range(T):
@@ -177,6 +179,27 @@ def test_explicit_calls_equal_step(B, flags):
             b.snapshot(); b.average_async()
     a.sync(); b.sync()
     assert torch.equal(a.w, b.w) and torch.equal(a.m, b.m)
+
+
+def test_inline_mean_needs_no_snapshot_arrays_and_refuses_delta(B):
+    K, P = 4, 5000
+    with pytest.raises(B.DasgdError) as e:
+        B.DaSGD(K, P, 2, 1, 0.25, merge_mode=1, flags=INLINE)
+    assert e.value.status == B.DASGD_ERR_INVALID_ARG
+    a = B.DaSGD(K, P, 2, 1, 0.25, 0.9, flags=INLINE, snapshot_arrays=False)
+    b = B.DaSGD(K, P, 2, 1, 0.25, 0.9)
+    assert a.snap is None
+    w0 = inputs.shared_start(21, P, 0.1)
+    a.set_state(w0); b.set_state(w0)
+    for t in range(11):
+        g = grads(22, t, K, P, 0.1, torch.float32, P)
+        a.step(g, 0.1); b.step(g, 0.1)
+    a.sync(); b.sync()
+    assert torch.equal(a.w, b.w) and torch.equal(a.m, b.m)
+    assert a.launches == 11                       # one kernel per iteration
+    with pytest.raises(B.DasgdError) as e:
+        a.snapshot()                               # the explicit calls need snapshot arrays
+    assert e.value.status in (B.DASGD_ERR_BAD_STATE, B.DASGD_ERR_NO_SLOT)
 
 
 def test_misuse_returns_status_codes(B):
