@@ -52,6 +52,28 @@ def step_bytes(wl):
 
 
 
+# DRAM traffic of one k_local_step_vec<f32, momentum> launch from an ncu capture on a smaller case
+# (K=8, P=4M; dram__bytes_read.sum + dram__bytes_write.sum = 384.0 + 205.2 MB for 32M updates); it grows
+# in proportion to K*P.  Valid only while the kernel source is the one that was profiled.
+NCU_TRAFFIC = {"kernels_sha256_prefix": "e38f2df3b9265ac4", "bytes_per_update": 589.2e6 / 32.0e6,
+               "applies_to": "float32 + momentum"}
+
+
+def profiled_traffic(wl):
+    """Bytes one local-step launch moves through DRAM according to the last ncu capture, or None when
+    the kernels have changed since, or the workload is not the profiled variant."""
+    import hashlib
+    try:
+        src = os.path.join(ROOT, "paper_2006_00441_b200", "csrc", "dasgd_kernels.cuh")
+        if hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] != NCU_TRAFFIC["kernels_sha256_prefix"]:
+            return None
+    except OSError:
+        return None
+    if wl.get("bf16") or not wl["momentum"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_update"] * wl["K"] * wl["P"]
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -384,7 +406,9 @@ def run_ours(args, wl, name):
                      "avg_launch_ms": (ms_step / n_step) if n_step else None,
                      "timed": f"CUDA events on the launching stream, instrumented pass of {n_inst} steps; the "
                               "side-stream mean kernel runs beside this kernel and shares HBM with it",
-                     "traffic": None,
+                     "traffic": profiled_traffic(wl),
+                     "traffic_note": "ncu dram bytes of a K=8, P=4M launch scaled by K*P; below the algorithmic "
+                                     "bytes because the last stores are still dirty in L2 when the kernel ends",
                      "alone": alone},
         "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
         "averaging_hidden_frac": hidden,
