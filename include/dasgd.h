@@ -180,6 +180,16 @@ dasgd_status dasgd_get_kernel_timing(dasgd_ctx *ctx, int32_t which, int64_t *n, 
 /* Synchronises and zeroes every timing counter. */
 dasgd_status dasgd_reset_timing(dasgd_ctx *ctx);
 
+/* Checkpointing.  The schedule state of a context (step counter, which array of the pool holds the
+ * current weights, the pending snapshots and their slots) as an opaque blob of at most 4096 bytes.
+ * dasgd_export_state synchronises both streams, then writes the blob to host_buf (*len receives its
+ * size; DASGD_ERR_INVALID_ARG if buf_len is too small).  To checkpoint, save the blob together with the
+ * contents of w, m, w_lp, snap and mean.  To resume, create a context with the same configuration
+ * over buffers holding the saved contents and call dasgd_import_state before any other call; the run
+ * then continues exactly as the original would have (the paper has no counterpart of these calls). */
+dasgd_status dasgd_export_state(dasgd_ctx *ctx, void *host_buf, int64_t buf_len, int64_t *len);
+dasgd_status dasgd_import_state(dasgd_ctx *ctx, const void *host_buf, int64_t len);
+
 /* Delay guideline of Section III-D (Eq. 3) and Section VI-C/VI-D: the averaging is fully hidden when
  * t_c < d * t_p (t_c: time of one averaging, t_p: time of one local update, same unit), so *d is the
  * smallest positive integer with that property and *tau = *d + 1.  Pure host arithmetic.

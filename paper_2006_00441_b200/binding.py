@@ -30,7 +30,7 @@ EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
     "dasgd_step", "dasgd_step_host", "dasgd_get_weights", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
-    "dasgd_average_merge_noalloc", "dasgd_delay_guideline", "dasgd_advise_delay",
+    "dasgd_average_merge_noalloc", "dasgd_delay_guideline", "dasgd_advise_delay", "dasgd_export_state", "dasgd_import_state",
 ]
 
 
@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     f64, pi32, pf64 = ctypes.c_double, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)
     L.dasgd_delay_guideline.argtypes = [f64, f64, pi32, pi32]
     L.dasgd_advise_delay.argtypes = [vp, f64, pi32, pi32, pf64, pf64]
+    L.dasgd_export_state.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
+    L.dasgd_import_state.argtypes = [vp, vp, i64]
     L.dasgd_version.argtypes = []
     L.dasgd_version.restype = ctypes.c_char_p
     return L
@@ -187,6 +189,16 @@ def dasgd_advise_delay(ctx, extra_tp_ms: float = 0.0):
     _check(_L.dasgd_advise_delay(ctx, extra_tp_ms, ctypes.byref(d), ctypes.byref(tau), ctypes.byref(tc),
                                  ctypes.byref(tp)), ctx)
     return d.value, tau.value, tc.value, tp.value
+
+
+def dasgd_export_state(ctx) -> bytes:
+    buf, n = ctypes.create_string_buffer(4096), ctypes.c_int64()
+    _check(_L.dasgd_export_state(ctx, buf, len(buf), ctypes.byref(n)), ctx)
+    return buf.raw[:n.value]
+
+
+def dasgd_import_state(ctx, blob: bytes):
+    _check(_L.dasgd_import_state(ctx, blob, len(blob)), ctx)
 
 
 def dasgd_get_launches(ctx) -> int:
@@ -352,6 +364,26 @@ class DaSGD:
 
     def reset_timing(self):
         dasgd_reset_timing(self.ctx)
+
+    def state_dict(self) -> dict:
+        """Everything needed to resume: the schedule blob and copies of the device arrays."""
+        blob = dasgd_export_state(self.ctx)       # synchronises both streams
+        out = {"schedule": blob, "w0": self._w0.clone(), "mean": self.mean.clone()}
+        for name in ("m", "w_lp", "snap"):
+            t = getattr(self, name)
+            out[name] = t.clone() if t is not None else None
+        torch.cuda.synchronize(self.device)
+        return out
+
+    def load_state_dict(self, sd: dict):
+        """Into a freshly built object of the same configuration."""
+        self.sync()
+        self._w0.copy_(sd["w0"]); self.mean.copy_(sd["mean"])
+        for name in ("m", "w_lp", "snap"):
+            if getattr(self, name) is not None and sd[name] is not None:
+                getattr(self, name).copy_(sd[name])
+        torch.cuda.synchronize(self.device)
+        dasgd_import_state(self.ctx, sd["schedule"])
 
     def advise_delay(self, extra_tp_ms=0.0):
         return dasgd_advise_delay(self.ctx, extra_tp_ms)

@@ -861,6 +861,83 @@ dasgd_status dasgd_reset_timing(dasgd_ctx *ctx) {
   return DASGD_OK;
 }
 
+namespace {
+struct StateHeader {
+  uint32_t magic, version;
+  int32_t K, tau, d, dtype, merge_mode, n_slots, pool, rotate;
+  int64_t P, ld, t;
+  int32_t cur, n_pending;
+};
+struct StatePending { int32_t slot, buf, state, pad; int64_t s; };
+constexpr uint32_t kStateMagic = 0x44615347u;  // "DaSG"
+}  // namespace
+
+dasgd_status dasgd_export_state(dasgd_ctx *ctx, void *host_buf, int64_t buf_len, int64_t *len) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!host_buf || !len) return fail(ctx, DASGD_ERR_INVALID_ARG, "export_state: NULL argument");
+  dasgd_status st = dasgd_sync(ctx);
+  if (st != DASGD_OK) return st;
+  const int64_t need = (int64_t)sizeof(StateHeader) + (int64_t)ctx->pending.size() * (int64_t)sizeof(StatePending);
+  *len = need;
+  if (buf_len < need) return fail(ctx, DASGD_ERR_INVALID_ARG, "export_state: buffer too small");
+  StateHeader h{};
+  h.magic = kStateMagic; h.version = 1;
+  h.K = ctx->cfg.K; h.tau = ctx->cfg.tau; h.d = ctx->cfg.d; h.dtype = ctx->cfg.dtype;
+  h.merge_mode = ctx->cfg.merge_mode; h.n_slots = ctx->cfg.n_slots; h.pool = (int32_t)ctx->pool.size();
+  h.rotate = ctx->rotate ? 1 : 0;
+  h.P = ctx->cfg.P; h.ld = ctx->cfg.ld; h.t = ctx->t;
+  h.cur = ctx->cur; h.n_pending = (int32_t)ctx->pending.size();
+  char *out = static_cast<char *>(host_buf);
+  std::memcpy(out, &h, sizeof h);
+  out += sizeof h;
+  for (int slot : ctx->pending) {
+    StatePending q{};
+    q.slot = slot; q.buf = ctx->slots[slot].buf; q.state = (int32_t)ctx->slots[slot].state; q.s = ctx->slots[slot].s;
+    std::memcpy(out, &q, sizeof q);
+    out += sizeof q;
+  }
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_import_state(dasgd_ctx *ctx, const void *host_buf, int64_t len) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!host_buf || len < (int64_t)sizeof(StateHeader)) return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: blob too short");
+  if (ctx->t != 0 || !ctx->pending.empty())
+    return fail(ctx, DASGD_ERR_BAD_STATE, "import_state: the context has already been used");
+  StateHeader h;
+  std::memcpy(&h, host_buf, sizeof h);
+  if (h.magic != kStateMagic || h.version != 1) return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: not a state blob");
+  const dasgd_config &c = ctx->cfg;
+  if (h.K != c.K || h.P != c.P || h.ld != c.ld || h.tau != c.tau || h.d != c.d || h.dtype != c.dtype ||
+      h.merge_mode != c.merge_mode || h.n_slots != c.n_slots || h.pool != (int32_t)ctx->pool.size() ||
+      h.rotate != (ctx->rotate ? 1 : 0))
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: the blob was exported from a different configuration");
+  if (h.n_pending < 0 || h.n_pending > c.n_slots || h.cur < 0 || h.cur >= h.pool || h.t < 0 ||
+      len < (int64_t)sizeof(StateHeader) + (int64_t)h.n_pending * (int64_t)sizeof(StatePending))
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: corrupt blob");
+  std::vector<StatePending> qs(h.n_pending);
+  if (h.n_pending) std::memcpy(qs.data(), static_cast<const char *>(host_buf) + sizeof h, qs.size() * sizeof(StatePending));
+  std::vector<bool> slot_seen(c.n_slots, false), buf_seen(ctx->pool.size(), false);
+  for (const StatePending &q : qs) {
+    if (q.slot < 0 || q.slot >= c.n_slots || slot_seen[q.slot] || q.buf < -1 || q.buf >= h.pool ||
+        (q.buf >= 0 && buf_seen[q.buf]) || (q.state != SLOT_SNAPPED && q.state != SLOT_AVERAGING))
+      return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: corrupt blob");
+    slot_seen[q.slot] = true;
+    if (q.buf >= 0) buf_seen[q.buf] = true;
+  }
+  ctx->t = h.t;
+  ctx->cur = h.cur;
+  for (const StatePending &q : qs) {
+    Slot &sl = ctx->slots[q.slot];
+    sl.state = (SlotState)q.state;   // the exporter had synchronised: a started mean is a finished mean,
+    sl.s = q.s;                      // so its (never recorded) event makes the later wait a no-op
+    sl.buf = q.buf;
+    if (q.buf >= 0) ctx->frozen[q.buf] = q.slot;
+    ctx->pending.push_back(q.slot);
+  }
+  return DASGD_OK;
+}
+
 dasgd_status dasgd_delay_guideline(double t_c, double t_p, int32_t *d, int32_t *tau) {
   if (!d || !tau || !(t_c >= 0.0) || !(t_p > 0.0)) return DASGD_ERR_INVALID_ARG;
   // d > t_c / t_p (Eq. 3): step up from the quotient so that rounding in the division cannot

@@ -66,3 +66,32 @@ def test_wrapper_refuses_to_run_without_a_gpu():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         B.DaSGD(2, 8, 1, 1, 0.25)
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/dasgd.h must compile as C99 on its own and every declared function must be linkable from C."""
+    import subprocess
+    src = tmp_path / "use_dasgd.c"
+    calls = "\n".join(f"  (void)&{n};" for n in declared_symbols())
+    src.write_text('#include "dasgd.h"\n#include <stddef.h>\nint main(void) {\n  dasgd_config c; c.K = 1; (void)c;\n'
+                   + calls + "\n  return (int)sizeof(dasgd_config) == 0;\n}\n")
+    exe = tmp_path / "use_dasgd"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"), str(src),
+                    B._build.LIB, "-Wl,-rpath," + os.path.dirname(B._build.LIB), "-o", str(exe)], check=True)
+    subprocess.run([str(exe)], check=True)
+
+
+def test_config_struct_layout_matches_the_binding(tmp_path):
+    """sizeof and field offsets of dasgd_config as the C compiler sees them == the ctypes mirror."""
+    import subprocess
+    fields = [f[0] for f in B.dasgd_config._fields_]
+    body = "\n".join(f'  printf("{f} %zu\\n", offsetof(dasgd_config, {f}));' for f in fields)
+    src = tmp_path / "layout.c"
+    src.write_text('#include "dasgd.h"\n#include <stddef.h>\n#include <stdio.h>\nint main(void) {\n'
+                   + body + '\n  printf("sizeof %zu\\n", sizeof(dasgd_config));\n  return 0;\n}\n')
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = dict(line.split() for line in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    for f in fields:
+        assert int(out[f]) == getattr(B.dasgd_config, f).offset, f
+    assert int(out["sizeof"]) == ctypes.sizeof(B.dasgd_config)

@@ -258,3 +258,52 @@ def test_timing_reports_hidden_fraction(B):
     assert all(v[1] > 0 for k, v in kt.items() if k != "stall")
     gpu.reset_timing()
     assert gpu.kernel_timing()["local_step"] == (0, 0.0)
+
+
+def test_sync_gives_up_after_its_timeout_and_the_context_survives(B):
+    """Failure detection on the host: dasgd_sync polls with a deadline.  Nothing on the GPU is made to
+    hang: the queue is simply longer than a 1 ms deadline."""
+    K, P = 8, 8_000_000
+    gpu = B.DaSGD(K, P, 1, 1, 0.25, 0.9, sync_timeout_ms=1, order_after_current=False)
+    g = torch.zeros(K, P, device="cuda")
+    torch.cuda.synchronize()
+    for _ in range(60):                       # tens of milliseconds of queued kernels
+        gpu.step(g, 0.1)
+    with pytest.raises(B.DasgdError) as e:
+        gpu.sync()
+    assert e.value.status == B.DASGD_ERR_TIMEOUT
+    torch.cuda.synchronize()                  # the work itself completes normally
+    gpu.sync()                                # and the context is still usable
+    gpu.step(g, 0.1)
+    torch.cuda.synchronize()
+    assert gpu.t == 61
+
+
+@pytest.mark.parametrize("tau,d,flags,mode", [(1, 1, ROTATE, 0), (1, 2, ROTATE | FUSE_MERGE, 0), (2, 3, 0, 1), (2, 1, FUSE_SNAP, 0),
+                                              (1, 2, ROTATE, 1), (2, 1, INLINE, 0)])
+def test_checkpoint_resume_continues_bit_for_bit(B, tau, d, flags, mode):
+    K, P, ld, T1, T2 = 3, 4096 + 40, 4096 + 40, 7, 6
+
+    def run(e, a, b):
+        for t in range(a, b):
+            e.step(grads(31, t, K, P, 0.05, torch.float32, ld), 0.1)
+
+    ref = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-3, merge_mode=mode, flags=flags)
+    ref.set_state(inputs.shared_start(30, P, 0.1))
+    run(ref, 0, T1)
+    sd = ref.state_dict()
+    run(ref, T1, T1 + T2)
+    ref.sync()
+    new = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-3, merge_mode=mode, flags=flags)
+    new.load_state_dict(sd)
+    snaps = list(range(tau, T1 + 1, tau))
+    assert new.t == T1 and new.n_pending == len([s for s in snaps if s + d > T1])
+    run(new, T1, T1 + T2)
+    new.sync()
+    assert new.t == ref.t
+    assert torch.equal(new.w[:, :P], ref.w[:, :P]) and torch.equal(new.m[:, :P], ref.m[:, :P])
+    with pytest.raises(B.DasgdError):
+        new.load_state_dict(sd)                   # only a fresh context may import
+    other = B.DaSGD(K, P, tau + 1, d, 0.25, 0.9, 1e-3, merge_mode=mode, flags=flags, n_slots=new.n_slots)
+    with pytest.raises(B.DasgdError):
+        other.load_state_dict(sd)                 # different configuration
