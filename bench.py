@@ -243,7 +243,7 @@ def run_ours(args, wl, name):
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
     torch.cuda.set_device(local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or args.force_dist:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
@@ -462,6 +462,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-fuse", action="store_true", help="run the unfused schedule (separate snapshot copy and merge)")
+    ap.add_argument("--force-dist", action="store_true",
+                    help="initialise the NCCL process group even with one rank (exercises the multi-rank plumbing)")
     ap.add_argument("--no-ablation", action="store_true", help="skip the inline-mean ablation leg")
     ap.add_argument("--sweep", action="store_true", help="run the K x tau x d sweep instead (one JSON line per point)")
     args = ap.parse_args()
