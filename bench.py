@@ -437,6 +437,77 @@ def run_sweep(args):
                     print(json.dumps(keep), flush=True)
 
 
+def run_mlp(args):
+    """End-to-end workload: K=8 replicas of a 4-layer, 4096-wide bf16 MLP trained against a fixed random
+    teacher (batch 256 per worker; forward/backward = batched bf16 matmuls of the GEMM library, on the
+    main stream), DaSGD update path with tau=1, d=1.  Here the averaging overlaps real compute."""
+    from paper_2006_00441_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    K, H, L, batch, lr, tau, d, xi = 8, 4096, 4, 256, 1e-3, 1, 1, 0.25
+    net = inputs.TeacherMLP(4, K, H, layers=L, batch=batch, device="cuda", dtype=torch.bfloat16)
+    net.precompute_batches(4)
+    P = net.P
+    flops_per_step = 3 * 2 * K * batch * H * H * L      # forward + two backward GEMMs per layer
+    out = {}
+    for name, flags in (("async", B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE | B.DASGD_FLAG_TIMING),
+                        ("inline_mean", B.DASGD_FLAG_INLINE_MEAN | B.DASGD_FLAG_TIMING)):
+        e = B.DaSGD(K, P, tau, d, xi, 0.9, 0.0, dtype=B.DASGD_BF16_MASTER_F32, flags=flags, order_after_current=False,
+                    snapshot_arrays=(name == "async"))
+        e.set_state(net.student_init())
+        g = torch.zeros(K, P, dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        losses = []
+        with torch.cuda.stream(e.main):
+            def one(t):
+                loss = net.forward_backward(t, e.w_lp, g)
+                e.step(g, lr)
+                return loss
+            for t in range(args.warmup):
+                one(t)
+            e.sync()
+            e.reset_timing()
+            l0 = e.launches
+            ev[0].record()
+            for t in range(args.steps):
+                loss = one(args.warmup + t)
+                if t in (0, args.steps - 1):
+                    losses.append(loss)
+            e.main.wait_stream(e.side)
+            ev[1].record()
+            # forward/backward alone, for the breakdown
+            e.sync()
+            for t in range(20):
+                net.forward_backward(t, e.w_lp, g)
+            ev[2].record()
+        e.sync()
+        torch.cuda.synchronize()
+        ms = ev[0].elapsed_time(ev[1]) / args.steps
+        ms_fb = ev[1].elapsed_time(ev[2]) / 20
+        kt = e.kernel_timing()
+        hidden = None
+        if kt["mean"][0] and kt["mean"][1] > 0:
+            hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
+        out[name] = {"value": K * P * args.steps / (ms * args.steps * 1e-3), "ms_per_step": ms,
+                     "ms_forward_backward": ms_fb, "gemm_tflops": flops_per_step / (ms_fb * 1e-3) / 1e12,
+                     "ms_update_path": ms - ms_fb, "gpu_launches": e.launches - l0, "averaging_hidden_frac": hidden,
+                     "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
+                     "loss_first_last": [float(x.mean()) for x in losses]}
+        e.close()
+        del e, g
+        torch.cuda.empty_cache()
+    line = {"metric": METRIC, "value": out["async"]["value"], "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": out["async"]["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/gradients/activations, f32 master", "data": "synthetic",
+            "config": {"workload": f"mlp: K={K} replicas of a {L}-layer {H}-wide bias-free ReLU MLP (P={P}), batch {batch} per "
+                                   f"worker, teacher-student regression, momentum 0.9, lr {lr}, tau={tau}, d={d}, xi={xi}",
+                       "K": K, "P": P, "tau": tau, "d": d, "xi": xi},
+            "async": out["async"], "inline_mean": out["inline_mean"]}
+    print(json.dumps(line), flush=True)
+
+
 def path_bytes_per_update(wl):
     """Algorithmic HBM bytes per replica-parameter update of the whole path as bench.py schedules it
     (rotating snapshots, merge folded into a step kernel when d >= 2): tau local steps, the snapshot
@@ -454,7 +525,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS) + ["mlp"])
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (profiling on a small case)")
     ap.add_argument("--K", type=int, default=0, help="override the number of replicas (sweep)")
     ap.add_argument("--tau", type=int, default=0, help="override the averaging period (sweep)")
@@ -469,7 +540,7 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    wl = dict(WORKLOADS[args.workload])
+    wl = dict(WORKLOADS.get(args.workload, {}))
     if args.P > 0:
         wl["P"] = args.P
     if args.K > 0:
@@ -478,7 +549,9 @@ def main():
         wl["tau"] = args.tau
     if args.d >= 0:
         wl["d"] = args.d
-    if args.sweep:
+    if args.workload == "mlp":
+        run_mlp(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args, wl, args.workload)
