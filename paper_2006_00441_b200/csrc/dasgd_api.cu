@@ -27,6 +27,7 @@ struct Slot {
   cudaEvent_t e_snap = nullptr;  // main stream: snapshot written
   cudaEvent_t e_avg = nullptr;   // side stream: mean written
   int buf = -1;                  // index into ctx->pool of the array that holds this snapshot
+  bool holds = false;            // this slot still keeps pool[buf] from being overwritten
 };
 
 // A pair of timing events around one piece of stream work, tagged with what it measures.
@@ -61,7 +62,8 @@ struct dasgd_ctx {
   std::vector<Slot> slots;
   std::deque<int> pending;  // slot indices, oldest snapshot first
   // Weight-sized arrays: pool[0] = cfg.w, pool[1 + i] = the i-th [K][ld] array of cfg.snap.
-  // `cur` holds the current weights; frozen[b] >= 0 names the pending slot whose snapshot is pool[b].
+  // `cur` holds the current weights; frozen[b] counts the pending slots whose snapshot is pool[b] (two
+  // snapshots taken with no weight update between them share one array).
   // Copy mode: cur stays 0 and snapshots are copies.  Rotate mode: a snapshot freezes `cur` itself and
   // the next kernel that writes weights writes them into a free array, which becomes `cur`.
   std::vector<float *> pool;
@@ -347,15 +349,24 @@ int find_free_slot(const dasgd_ctx *c) {
 // An array that is neither the current weights nor a pending snapshot; `fallback` (or -1) otherwise.
 int find_free_buf(const dasgd_ctx *c, int fallback) {
   for (size_t b = 0; b < c->pool.size(); ++b)
-    if ((int)b != c->cur && c->frozen[b] < 0) return (int)b;
+    if ((int)b != c->cur && c->frozen[b] == 0) return (int)b;
   return fallback;
+}
+
+// The snapshot array of `slot` if the kernel that merges that slot may overwrite it element by element
+// (nobody else still needs it), else -1.
+int reusable_buf(const dasgd_ctx *c, int slot) {
+  const Slot &sl = c->slots[slot];
+  if (sl.buf < 0) return -1;
+  const int others = c->frozen[sl.buf] - (sl.holds ? 1 : 0);
+  return others == 0 ? sl.buf : -1;
 }
 
 // Where the next kernel that writes weights must put them: in place unless the current array is a
 // pending snapshot.  `reusable` is an array the same kernel is allowed to overwrite element by
 // element after reading it (the snapshot of the slot it merges), or -1.
 int pick_w_out(const dasgd_ctx *c, int reusable) {
-  if (c->frozen[c->cur] < 0) return c->cur;
+  if (c->frozen[c->cur] == 0) return c->cur;
   return find_free_buf(c, reusable);
 }
 
@@ -366,7 +377,8 @@ dasgd_status mark_snapped(dasgd_ctx *c, int slot, int buf) {
   sl.state = SLOT_SNAPPED;
   sl.s = c->t;
   sl.buf = buf;
-  c->frozen[buf] = slot;
+  c->frozen[buf] += 1;
+  sl.holds = true;
   c->pending.push_back(slot);
   return DASGD_OK;
 }
@@ -383,7 +395,10 @@ dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
   span_end(c, sp, c->s0);
   // From here on the main stream is ordered after the mean kernel.  The xi-blend no longer needs
   // the snapshot itself, so its array may be overwritten by what the main stream does next.
-  if (c->cfg.merge_mode == DASGD_MERGE_XI && sl.buf >= 0) c->frozen[sl.buf] = -1;
+  if (c->cfg.merge_mode == DASGD_MERGE_XI && sl.holds) {
+    c->frozen[sl.buf] -= 1;
+    sl.holds = false;
+  }
   *slot_out = slot;
   return DASGD_OK;
 }
@@ -392,7 +407,10 @@ void release_oldest(dasgd_ctx *c) {
   const int slot = c->pending.front();
   c->pending.pop_front();
   Slot &sl = c->slots[slot];
-  if (sl.buf >= 0 && c->frozen[sl.buf] == slot) c->frozen[sl.buf] = -1;
+  if (sl.holds) {
+    c->frozen[sl.buf] -= 1;
+    sl.holds = false;
+  }
   sl.state = SLOT_FREE;
 }
 
@@ -498,7 +516,7 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   ctx->pool.push_back(static_cast<float *>(c.w));
   for (int i = 0; c.snap && i < c.n_slots; ++i)
     ctx->pool.push_back(static_cast<float *>(c.snap) + (size_t)i * c.K * c.ld);
-  ctx->frozen.assign(ctx->pool.size(), -1);
+  ctx->frozen.assign(ctx->pool.size(), 0);
   DeviceGuard guard(c.device);
   ctx->slots.resize(c.n_slots);
   for (Slot &sl : ctx->slots) {
@@ -566,7 +584,7 @@ dasgd_status op_step(dasgd_ctx *c, const void *grads, float lr, int merge_slot, 
   if (merge_slot >= 0) {
     p.mean = mean_ptr(c, merge_slot);
     p.snap_in = snap_ptr(c, merge_slot);
-    reusable = c->slots[merge_slot].buf;
+    reusable = reusable_buf(c, merge_slot);
   }
   const int out = pick_w_out(c, reusable);
   if (out < 0) return fail(c, DASGD_ERR_NO_SLOT, "step: no free weight array to write into");
@@ -585,7 +603,7 @@ dasgd_status op_merge(dasgd_ctx *c, int slot, int snap_buf) {
   Params p = base_params(c);
   p.mean = mean_ptr(c, slot);
   p.snap_in = snap_ptr(c, slot);
-  const int out = pick_w_out(c, c->slots[slot].buf);
+  const int out = pick_w_out(c, reusable_buf(c, slot));
   if (out < 0) return fail(c, DASGD_ERR_NO_SLOT, "merge: no free weight array to write into");
   p.w_out = c->pool[out];
   if (snap_buf >= 0) p.snap_out = c->pool[snap_buf];
@@ -617,7 +635,7 @@ dasgd_status op_snapshot(dasgd_ctx *c, int already_in) {
 // One iteration of the inline-mean schedule: everything on the main stream, one kernel (two when
 // d == 0, because the blend then needs the mean of the very weights this kernel produces).
 dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, bool s_due) {
-  if (c->frozen[c->cur] >= 0)
+  if (c->frozen[c->cur] > 0)
     return fail(c, DASGD_ERR_BAD_STATE, "step: a snapshot taken with dasgd_snapshot is pending; merge it first");
   Params p = base_params(c);
   p.g = grads;
@@ -647,6 +665,7 @@ dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, 
     sl.state = SLOT_AVERAGING;  // the mean is already on its way, on this same stream
     sl.s = c->t;
     sl.buf = -1;                // no snapshot array belongs to it
+    sl.holds = false;
     c->pending.push_back(slot);
     if (c->cfg.d == 0) {        // Local SGD: blend it back at once
       Params q = base_params(c);
@@ -716,7 +735,7 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
   if (fuse_snap && (!m_due || fuse_merge)) {
     // A kernel that merges a slot may store the new snapshot over that slot's old one: each thread
     // reads the old element before it writes the new one.
-    stored_in = find_free_buf(ctx, merge_slot >= 0 ? ctx->slots[merge_slot].buf : -1);
+    stored_in = find_free_buf(ctx, merge_slot >= 0 ? reusable_buf(ctx, merge_slot) : -1);
     if (stored_in < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot array");
   }
   st = op_step(ctx, grads, lr, merge_slot, stored_in);
@@ -728,7 +747,7 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
     st = wait_oldest_average(ctx, &merge_slot);
     if (st != DASGD_OK) return st;
     if (fuse_snap) {
-      stored_in = find_free_buf(ctx, ctx->slots[merge_slot].buf);
+      stored_in = find_free_buf(ctx, reusable_buf(ctx, merge_slot));
       if (stored_in < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot array");
     }
     st = op_merge(ctx, merge_slot, stored_in);
@@ -917,13 +936,12 @@ dasgd_status dasgd_import_state(dasgd_ctx *ctx, const void *host_buf, int64_t le
     return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: corrupt blob");
   std::vector<StatePending> qs(h.n_pending);
   if (h.n_pending) std::memcpy(qs.data(), static_cast<const char *>(host_buf) + sizeof h, qs.size() * sizeof(StatePending));
-  std::vector<bool> slot_seen(c.n_slots, false), buf_seen(ctx->pool.size(), false);
+  std::vector<bool> slot_seen(c.n_slots, false);
   for (const StatePending &q : qs) {
     if (q.slot < 0 || q.slot >= c.n_slots || slot_seen[q.slot] || q.buf < -1 || q.buf >= h.pool ||
-        (q.buf >= 0 && buf_seen[q.buf]) || (q.state != SLOT_SNAPPED && q.state != SLOT_AVERAGING))
+        (q.state != SLOT_SNAPPED && q.state != SLOT_AVERAGING))
       return fail(ctx, DASGD_ERR_INVALID_ARG, "import_state: corrupt blob");
     slot_seen[q.slot] = true;
-    if (q.buf >= 0) buf_seen[q.buf] = true;
   }
   ctx->t = h.t;
   ctx->cur = h.cur;
@@ -932,7 +950,8 @@ dasgd_status dasgd_import_state(dasgd_ctx *ctx, const void *host_buf, int64_t le
     sl.state = (SlotState)q.state;   // the exporter had synchronised: a started mean is a finished mean,
     sl.s = q.s;                      // so its (never recorded) event makes the later wait a no-op
     sl.buf = q.buf;
-    if (q.buf >= 0) ctx->frozen[q.buf] = q.slot;
+    sl.holds = q.buf >= 0;
+    if (sl.holds) ctx->frozen[q.buf] += 1;
     ctx->pending.push_back(q.slot);
   }
   return DASGD_OK;

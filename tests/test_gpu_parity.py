@@ -307,3 +307,43 @@ def test_checkpoint_resume_continues_bit_for_bit(B, tau, d, flags, mode):
     other = B.DaSGD(K, P, tau + 1, d, 0.25, 0.9, 1e-3, merge_mode=mode, flags=flags, n_slots=new.n_slots)
     with pytest.raises(B.DasgdError):
         other.load_state_dict(sd)                 # different configuration
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("flags,mode", [(0, 0), (ROTATE, 0), (ROTATE, 1), (0, 1)])
+def test_random_call_sequences_match_the_oracle(B, seed, flags, mode):
+    """Scheduler fuzz: random but valid orders of the four explicit calls (several snapshots in flight,
+    means started late, merges in bursts), the same order on the library and on the oracle."""
+    import random
+    rnd = random.Random(seed * 7 + flags + mode)
+    K, P, n_slots = rnd.choice([2, 3, 5]), rnd.choice([1000, 4096 + 9, 2 * 4096]), 3
+    ld = (P + 7) // 8 * 8
+    gpu, cpu = make_pair(B, K, P, 1, n_slots, 0.25, 0.9, 1e-3, merge_mode=mode, flags=flags, ld=ld, n_slots=n_slots,
+                         w0=inputs.shared_start(40 + seed, P, 0.1).numpy())
+    snapped = averaged = 0          # snapshots without a mean yet / with a mean, oldest first overall
+    for i in range(60):
+        choices = ["step"]
+        if snapped + averaged < n_slots:
+            choices.append("snapshot")
+        if snapped:
+            choices.append("average")
+        if averaged and snapped + averaged > 0:
+            choices.append("merge")
+        op = rnd.choice(choices)
+        if op == "step":
+            g = grads(41 + seed, i, K, P, 0.05, torch.float32, ld)
+            gpu.local_step(g, 0.1); cpu.local_step(to_oracle_grad(g, P), 0.1)
+        elif op == "snapshot":
+            gpu.snapshot(); cpu.snapshot(); snapped += 1
+        elif op == "average":
+            gpu.average_async(); cpu.average(); snapped -= 1; averaged += 1
+        else:
+            # the oldest pending snapshot must be the one that has its mean: true because means are
+            # started oldest first and merged oldest first
+            gpu.merge(); cpu.merge(); averaged -= 1
+        assert gpu.n_pending == cpu.n_pending == snapped + averaged
+    w, m = state_of(gpu)
+    assert_close(w, cpu.w, TOL_RUN, "w"); assert_close(m, cpu.m, TOL_RUN, "m")
+    for j in range(averaged):
+        _, _, mean = cpu.pending(j)
+        assert_close(gpu.pending_mean(j).cpu().numpy(), mean, TOL_RUN, f"mean {j}")
