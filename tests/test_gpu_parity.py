@@ -347,3 +347,35 @@ def test_random_call_sequences_match_the_oracle(B, seed, flags, mode):
     for j in range(averaged):
         _, _, mean = cpu.pending(j)
         assert_close(gpu.pending_mean(j).cpu().numpy(), mean, TOL_RUN, f"mean {j}")
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_configurations_match_the_oracle(B, seed):
+    """Random draws over every knob of dasgd_step (sizes, schedule, hyper-parameters, dtype, merge form,
+    fusion flags, extra slots), 40 steps each."""
+    import random
+    rnd = random.Random(1000 + seed)
+    K = rnd.choice([1, 2, 3, 4, 7, 8, 9, 16, 31])
+    P = rnd.choice([1, 5, 8, 63, 1000, 4095, 4096, 4097, 9000, 3 * 4096 + 5])
+    tau, d = rnd.choice([1, 2, 3, 5]), rnd.choice([0, 1, 1, 2, 3, 4])
+    xi = rnd.choice([0.0, 0.25, 0.5, 0.9, 1.0])
+    mom, wd = rnd.choice([0.0, 0.5, 0.9]), rnd.choice([0.0, 1e-4, 1e-2])
+    dtype, mode = rnd.choice([0, 0, 1]), rnd.choice([0, 0, 1])
+    flags = rnd.choice([0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE] + ([INLINE] if mode == 0 else []))
+    ld = rnd.choice([P, (P + 7) // 8 * 8, (P + 7) // 8 * 8 + 8])
+    n_slots = max(1, -(-d // tau)) + rnd.choice([0, 0, 1])
+    gd = torch.bfloat16 if dtype else torch.float32
+    gpu, cpu = make_pair(B, K, P, tau, d, xi, mom, wd, dtype=dtype, merge_mode=mode, flags=flags, ld=ld, n_slots=n_slots,
+                         w0=inputs.shared_start(seed, P, 0.05).numpy())
+    lr = rnd.choice([0.01, 0.1])
+    for t in range(40):
+        g = grads(2000 + seed, t, K, P, 0.05, gd, ld)
+        gpu.step(g, lr); cpu.step(to_oracle_grad(g, P), lr)
+        assert gpu.n_pending == cpu.n_pending
+    w, m = state_of(gpu)
+    what = f"K={K} P={P} ld={ld} tau={tau} d={d} xi={xi} mom={mom} wd={wd} dtype={dtype} mode={mode} flags={flags} slots={n_slots}"
+    assert_close(w, cpu.w, TOL_RUN, what)
+    if mom:
+        assert_close(m, cpu.m, TOL_RUN, what)
+    if dtype:
+        np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), bf16_bits(gpu.w[:, :P].to(torch.bfloat16)))
