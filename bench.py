@@ -340,6 +340,12 @@ def run_ours(args, wl, name):
     if kt["mean"][0] and kt["mean"][1] > 0:
         hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
 
+    hidden_cost = None
+    if all(k in alone for k in ("local_step", "mean", "merge")):
+        tau_, d_ = wl["tau"], wl["d"]
+        main_alone = tau_ * alone["local_step"]["ms"] + (alone["merge"]["ms"] if d_ < 2 else 0.0)
+        hidden_cost = 1.0 - (ms / args.steps * tau_ - main_alone) / alone["mean"]["ms"]
+
     # ---- ablation: the same work with the mean computed inside the step kernel (no side stream)
     ablation = None
     if not args.no_ablation:
@@ -412,6 +418,12 @@ def run_ours(args, wl, name):
                      "alone": alone},
         "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
         "averaging_hidden_frac": hidden,
+        "averaging_hidden_frac_cost": hidden_cost,
+        "averaging_hidden_note": "averaging_hidden_frac: share of the mean kernel's time during which the main stream "
+                                 "did not wait for it (the paper's notion: the critical path never stalls).  "
+                                 "_cost: 1 - (cycle time - cycle time of the main-stream kernels alone) / mean kernel "
+                                 "alone; on one GPU the mean competes with the local step for the same HBM, so its "
+                                 "bytes are not free even though nothing waits for it",
         "whole_path_gbs": value / world * path_bytes_per_update(wl) / 1e9,
         "ablation_inline_mean": ablation,
         "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
