@@ -226,11 +226,12 @@ def test_misuse_returns_status_codes(B):
     assert gpu.t == 1
 
 
+@pytest.mark.parametrize("flags", [0, ROTATE | FUSE_MERGE, INLINE])
 @pytest.mark.parametrize("n_stage", [1, 2])
-def test_step_host_matches_step(B, n_stage):
+def test_step_host_matches_step(B, n_stage, flags):
     K, P, T = 4, 4096 + 8, 9
     w0 = inputs.shared_start(8, P, 0.1)
-    a = B.DaSGD(K, P, 2, 1, 0.25, 0.9, host_staging=n_stage)
+    a = B.DaSGD(K, P, 2, 1, 0.25, 0.9, host_staging=n_stage, flags=flags)
     b = B.DaSGD(K, P, 2, 1, 0.25, 0.9)
     a.set_state(w0); b.set_state(w0)
     probe = torch.empty(256, dtype=torch.float32).pin_memory()
