@@ -79,6 +79,12 @@ typedef enum {
                                          mean is no longer computed asynchronously.  xi-blend merge only.  The
                                          explicit snapshot/average/merge calls keep working if snap is given. */
 
+/* Variants of the local step.  The paper names only "weight decay 0.01, moment 0.9" on its platform
+ * (Section IV-A) and gives no formula, so the common forms are all offered; the default is the plain one. */
+#define DASGD_FLAG_NESTEROV 0x20u      /* w <- w - lr*(g' + mu*m) with the freshly updated m (needs momentum > 0) */
+#define DASGD_FLAG_DECOUPLED_WD 0x40u  /* g' = g, and w <- w - lr*lambda*w - lr*(step direction): the decay acts
+                                          on the weights directly instead of entering the momentum            */
+
 typedef struct dasgd_config {
   int32_t K;            /* workers (the paper's M), >= 1                                              */
   int32_t tau;          /* local steps between snapshots, >= 1                                        */

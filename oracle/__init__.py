@@ -58,6 +58,7 @@ def bind(path: str) -> ctypes.CDLL:
     L.oracle_dasgd_average.argtypes = [vp]
     L.oracle_dasgd_merge.argtypes = [vp]
     L.oracle_dasgd_step.argtypes = [vp, vp, f32]
+    L.oracle_dasgd_set_variant.argtypes = [vp, i32, i32]
     L.oracle_dasgd_threads.argtypes = []
     f64, pi32 = ctypes.c_double, ctypes.POINTER(i32)
     L.oracle_dasgd_delay_guideline.argtypes = [f64, f64, pi32, pi32]
@@ -99,12 +100,14 @@ class OracleDaSGD:
     """K replicas of a P-vector driven by the oracle.  Arrays are numpy, [K][P]."""
 
     def __init__(self, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=F32,
-                 merge_mode=MERGE_XI, omp=False):
+                 merge_mode=MERGE_XI, omp=False, nesterov=False, decoupled_wd=False):
         self._L = _lib(omp)
         self.K, self.P, self.tau, self.d, self.dtype = K, P, tau, d, dtype
         self._h = self._L.oracle_dasgd_create(K, P, tau, d, xi, momentum, weight_decay, dtype, merge_mode)
         if not self._h:
             raise OracleError("invalid configuration")
+        if (nesterov or decoupled_wd) and self._L.oracle_dasgd_set_variant(self._h, int(nesterov), int(decoupled_wd)) != 0:
+            raise OracleError("invalid variant (Nesterov needs momentum)")
 
     def close(self):
         if getattr(self, "_h", None):

@@ -45,6 +45,7 @@ struct oracle_dasgd {
   int32_t K, tau, d, dtype, merge_mode;
   int64_t P;
   float xi, momentum, weight_decay;
+  bool nesterov = false, decoupled_wd = false;
   int64_t t;  // completed local steps
   std::vector<float> w, m;
   std::vector<uint16_t> w_lp;
@@ -72,6 +73,13 @@ oracle_dasgd *oracle_dasgd_create(int32_t K, int64_t P, int32_t tau, int32_t d, 
 }
 
 void oracle_dasgd_destroy(oracle_dasgd *o) { delete o; }
+
+int oracle_dasgd_set_variant(oracle_dasgd *o, int32_t nesterov, int32_t decoupled_wd) {
+  if (!o || (nesterov && o->momentum == 0.0f)) return ORACLE_ERR_ARG;
+  o->nesterov = nesterov != 0;
+  o->decoupled_wd = decoupled_wd != 0;
+  return ORACLE_OK;
+}
 
 int oracle_dasgd_set_state(oracle_dasgd *o, const float *w, const float *m) {
   if (!o || !w) return ORACLE_ERR_ARG;
@@ -126,13 +134,15 @@ int oracle_dasgd_local_step(oracle_dasgd *o, const void *g, float lr) {
     for (int64_t p = 0; p < P; ++p) {
       const size_t i = static_cast<size_t>(k) * P + p;
       const double gi = bf16 ? static_cast<double>(bf16_to_f32(g16[i])) : static_cast<double>(g32[i]);
-      const double gp = gi + lambda * static_cast<double>(o->w[i]);
+      const double w_old = o->w[i];
+      const double gp = o->decoupled_wd ? gi : gi + lambda * w_old;
+      double dir = gp;  // the direction the weights move along
       if (o->momentum != 0.0f) {
         o->m[i] = static_cast<float>(mu * static_cast<double>(o->m[i]) + gp);
-        o->w[i] = static_cast<float>(static_cast<double>(o->w[i]) - eta * static_cast<double>(o->m[i]));
-      } else {
-        o->w[i] = static_cast<float>(static_cast<double>(o->w[i]) - eta * gp);
+        dir = o->nesterov ? gp + mu * static_cast<double>(o->m[i]) : static_cast<double>(o->m[i]);
       }
+      const double decay = o->decoupled_wd ? eta * lambda * w_old : 0.0;
+      o->w[i] = static_cast<float>(w_old - decay - eta * dir);
       if (bf16) o->w_lp[i] = f32_to_bf16_rne(o->w[i]);
     }
   }

@@ -56,6 +56,11 @@ oracle_dasgd *oracle_dasgd_create(int32_t K, int64_t P, int32_t tau, int32_t d, 
                                   float momentum, float weight_decay, int32_t dtype,
                                   int32_t merge_mode);
 void oracle_dasgd_destroy(oracle_dasgd *o);
+/* Variants of the local step (the paper gives no formula, Section IV-A names only the values):
+ *   nesterov:      w <- w - eta*(g' + mu*m) with the freshly updated m   (pinned: torch.optim.SGD(nesterov=True))
+ *   decoupled_wd:  g' = g and w <- w - eta*lambda*w - eta*(step direction) (pinned: w*(1-eta*lambda) followed by
+ *                  torch.optim.SGD without weight decay, and the closed form (1-eta*lambda)^T for zero gradients) */
+int oracle_dasgd_set_variant(oracle_dasgd *o, int32_t nesterov, int32_t decoupled_wd);
 
 /* State access: w, m are [K][P] float32 (row k = worker k); w_lp is [K][P] bf16 bits. */
 int oracle_dasgd_set_state(oracle_dasgd *o, const float *w, const float *m);

@@ -25,6 +25,7 @@ DASGD_F32, DASGD_BF16_MASTER_F32 = 0, 1
 DASGD_MERGE_XI, DASGD_MERGE_DELTA = 0, 1
 DASGD_FLAG_TIMING, DASGD_FLAG_FUSE_SNAPSHOT, DASGD_FLAG_FUSE_MERGE, DASGD_FLAG_ROTATE_SNAPSHOT = 0x1, 0x2, 0x4, 0x8
 DASGD_FLAG_INLINE_MEAN = 0x10
+DASGD_FLAG_NESTEROV, DASGD_FLAG_DECOUPLED_WD = 0x20, 0x40
 
 EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",

@@ -117,6 +117,8 @@ Params base_params(const dasgd_ctx *c) {
   p.K = c->cfg.K;
   p.mu = c->cfg.momentum;
   p.lambda = c->cfg.weight_decay;
+  p.nesterov = (c->cfg.flags & DASGD_FLAG_NESTEROV) ? 1 : 0;
+  p.decoupled_wd = (c->cfg.flags & DASGD_FLAG_DECOUPLED_WD) ? 1 : 0;
   p.xi = c->cfg.xi;
   p.omx = 1.0f - c->cfg.xi;
   return p;
@@ -482,6 +484,8 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   const int need = c.d == 0 ? 1 : (c.d + c.tau - 1) / c.tau;
   if (c.n_slots < need)
     return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: n_slots must be >= max(1, ceil(d/tau))");
+  if ((c.flags & DASGD_FLAG_NESTEROV) && c.momentum == 0.0f)
+    return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: DASGD_FLAG_NESTEROV needs momentum > 0");
   const bool inline_mean = (c.flags & DASGD_FLAG_INLINE_MEAN) != 0;
   if (inline_mean && c.merge_mode != DASGD_MERGE_XI)
     return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: DASGD_FLAG_INLINE_MEAN supports the xi-blend merge only");

@@ -13,6 +13,8 @@
 // Arithmetic is float32 with explicit fused multiply-adds, the same expressions in every
 // variant, so that fused and unfused schedules give bit-identical results:
 //     g' = fma(lambda, w, g);  m = fma(mu, m, g');  w = fma(-lr, m, w)        (local step)
+//       Nesterov:            w = fma(-lr, fma(mu, m, g'), w)
+//       decoupled decay:     g' = g;  w = fma(-(lr*lambda), w_old, fma(-lr, dir, w_old))
 //     w  = fma(xi, w, (1-xi)*mean)                                            (xi merge)
 //     w  = w + (mean - snap)                                                  (delta merge)
 //     mean = (pairwise sum over k) / K                                        (worker-axis mean)
@@ -39,6 +41,8 @@ struct Params {
   long long P, ld;
   int K;
   float lr, mu, lambda, xi, omx;
+  int nesterov;      // 1: step along g' + mu*m instead of m
+  int decoupled_wd;  // 1: weight decay is applied to the weights directly, not added to the gradient
 };
 
 // ---------------------------------------------------------------- memory helpers
@@ -60,13 +64,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 template <bool MOM>
 __device__ __forceinline__ void step_elem(float &w, float &m, float g, const Params &p) {
-  const float gp = fmaf(p.lambda, w, g);
+  // the two variant switches are uniform across the grid, so the branches cost nothing here
+  const float gp = p.decoupled_wd ? g : fmaf(p.lambda, w, g);
+  float dir = gp;
   if (MOM) {
     m = fmaf(p.mu, m, gp);
-    w = fmaf(-p.lr, m, w);
-  } else {
-    w = fmaf(-p.lr, gp, w);
+    dir = p.nesterov ? fmaf(p.mu, m, gp) : m;
   }
+  const float w_old = w;
+  w = fmaf(-p.lr, dir, w);
+  if (p.decoupled_wd) w = fmaf(-__fmul_rn(p.lr, p.lambda), w_old, w);
 }
 
 __device__ __forceinline__ float blend_xi(float w, float mean, const Params &p) {

@@ -39,7 +39,8 @@ def make_pair(B, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=0, merg
     """A libdasgd instance and an oracle with the same configuration and start point."""
     gpu = B.DaSGD(K, P, tau, d, xi, momentum, weight_decay, dtype=dtype, merge_mode=merge_mode, flags=flags,
                   ld=ld, n_slots=n_slots)
-    cpu = OracleDaSGD(K, P, tau, d, xi, momentum, weight_decay, dtype=dtype, merge_mode=merge_mode)
+    cpu = OracleDaSGD(K, P, tau, d, xi, momentum, weight_decay, dtype=dtype, merge_mode=merge_mode,
+                      nesterov=bool(flags & 0x20), decoupled_wd=bool(flags & 0x40))
     if w0 is not None:
         w0 = np.asarray(w0, np.float32)
         gpu.set_state(torch.from_numpy(w0))

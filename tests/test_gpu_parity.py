@@ -14,6 +14,7 @@ from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, make_pair,
 pytestmark = pytest.mark.gpu
 
 FUSE_SNAP, FUSE_MERGE, ROTATE, INLINE = 0x2, 0x4, 0x8, 0x10
+NESTEROV, DECOUPLED = 0x20, 0x40
 # f32 vector tile = 256 threads * 4 units * 4 elements = 4096 elements; bf16 tile = 256*2*8 = 4096
 SIZES = [1, 3, 4, 7, 8, 1000, 4096, 3 * 4096 + 1029]
 
@@ -83,6 +84,38 @@ def test_snapshot_mean_merge_teacher_forced(B, P, K, dtype, mode):
     if dtype:
         np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), bf16_bits(gpu.w[:, :P].to(torch.bfloat16)))
     assert gpu.n_pending == 0 and cpu.n_pending == 0
+
+
+@pytest.mark.parametrize("variant", [NESTEROV, DECOUPLED, NESTEROV | DECOUPLED])
+@pytest.mark.parametrize("sched", [0, ROTATE | FUSE_MERGE, INLINE])
+@pytest.mark.parametrize("dtype,P", [(0, 4096 + 7), (1, 2 * 4096 + 9), (0, 5)])
+def test_local_step_variants(B, variant, sched, dtype, P):
+    """Nesterov momentum and decoupled weight decay: one teacher-forced step at 1e-6, then 60 free steps."""
+    K, ld = 3, (P + 7) // 8 * 8
+    gd = torch.bfloat16 if dtype else torch.float32
+    w0 = inputs.shared_start(50, P, 0.5).numpy()
+    gpu, cpu = make_pair(B, K, P, 2, 2, 0.25, 0.9, 0.05, dtype=dtype, flags=variant | sched, ld=ld, w0=w0)
+    g = grads(51, 0, K, P, 0.3, gd, ld)
+    gpu.local_step(g, 0.1); cpu.local_step(to_oracle_grad(g, P), 0.1)
+    w, m = state_of(gpu)
+    assert_close(w, cpu.w, TOL_STEP, "w after one step"); assert_close(m, cpu.m, TOL_STEP, "m after one step")
+    gpu2, cpu2 = make_pair(B, K, P, 2, 2, 0.25, 0.9, 0.05, dtype=dtype, flags=variant | sched, ld=ld, w0=w0)
+    for t in range(60):
+        g = grads(52, t, K, P, 0.1, gd, ld)
+        gpu2.step(g, 0.05); cpu2.step(to_oracle_grad(g, P), 0.05)
+    w, m = state_of(gpu2)
+    assert_close(w, cpu2.w, TOL_RUN, "w"); assert_close(m, cpu2.m, TOL_RUN, "m")
+    plain, _ = make_pair(B, K, P, 2, 2, 0.25, 0.9, 0.05, dtype=dtype, flags=sched, ld=ld, w0=w0)
+    for t in range(60):
+        plain.step(grads(52, t, K, P, 0.1, gd, ld), 0.05)
+    wp, _ = state_of(plain)
+    assert np.abs(wp - w).max() > 1e-4            # the variants really change the trajectory
+
+
+def test_nesterov_needs_momentum(B):
+    with pytest.raises(B.DasgdError) as e:
+        B.DaSGD(2, 64, 2, 1, 0.25, 0.0, flags=NESTEROV)
+    assert e.value.status == B.DASGD_ERR_INVALID_ARG
 
 
 # ------------------------------------------------------------------ free-running schedules

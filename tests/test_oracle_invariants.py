@@ -267,6 +267,66 @@ def test_weight_decay_closed_form_zero_gradient():
     assert np.all(o.w == np.float32(8.0 * (1 - lr * wd) ** T))
 
 
+# ------------------------------------------------------------------ variants of the local step
+
+def _torch_sgd_run(w0, G, lr, mu, wd, nesterov=False, scale_weights_by=None):
+    p = torch.tensor(w0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([p], lr=float(np.float32(lr)), momentum=float(np.float32(mu)),
+                          weight_decay=float(np.float32(wd)), nesterov=nesterov)
+    for t in range(G.shape[0]):
+        if scale_weights_by is not None:
+            with torch.no_grad():
+                p.mul_(scale_weights_by)
+        p.grad = torch.tensor(G[t], dtype=torch.float64)
+        opt.step()
+    return p.detach().numpy()
+
+
+def test_nesterov_matches_torch():
+    K, P, T, lr, mu, wd = 2, 23, 12, 0.1, 0.9, 0.01
+    G = rng_grads(T, K, P, 30)
+    w0 = np.random.default_rng(31).standard_normal((K, P)).astype(np.float32)
+    o = OracleDaSGD(K, P, 3, 1, xi=1.0, momentum=mu, weight_decay=wd, nesterov=True)
+    o.set_state(w0)
+    for t in range(T):
+        o.step(G[t], lr)
+    np.testing.assert_allclose(o.w, _torch_sgd_run(w0, G, lr, mu, wd, nesterov=True), rtol=3e-6, atol=3e-6)
+    plain = OracleDaSGD(K, P, 3, 1, xi=1.0, momentum=mu, weight_decay=wd)
+    plain.set_state(w0)
+    for t in range(T):
+        plain.step(G[t], lr)
+    assert np.abs(plain.w - o.w).max() > 1e-3          # the variant is not a no-op
+
+
+@pytest.mark.parametrize("mu,nesterov", [(0.9, False), (0.0, False), (0.5, True)])
+def test_decoupled_weight_decay_matches_scaled_weights_then_torch(mu, nesterov):
+    """w <- w - eta*lambda*w - eta*dir  ==  scale the weights by (1 - eta*lambda), then an SGD step without decay."""
+    K, P, T, lr, wd = 2, 19, 10, 0.1, 0.05
+    G = rng_grads(T, K, P, 32)
+    w0 = np.random.default_rng(33).standard_normal((K, P)).astype(np.float32)
+    o = OracleDaSGD(K, P, 2, 1, xi=1.0, momentum=mu, weight_decay=wd, decoupled_wd=True, nesterov=nesterov)
+    o.set_state(w0)
+    for t in range(T):
+        o.step(G[t], lr)
+    scale = 1.0 - float(np.float32(lr)) * float(np.float32(wd))
+    want = _torch_sgd_run(w0, G, lr, mu, 0.0, nesterov=nesterov, scale_weights_by=scale)
+    np.testing.assert_allclose(o.w, want, rtol=3e-6, atol=3e-6)
+
+
+def test_decoupled_weight_decay_closed_form_with_momentum():
+    """Zero gradients: decoupled decay shrinks w by (1 - eta*lambda) per step whatever the momentum
+    (the coupled form would not, because the decay term accumulates in the momentum buffer)."""
+    lr, wd, T = 0.5, 0.25, 6
+    o = OracleDaSGD(1, 2, 2, 1, xi=1.0, momentum=0.9, weight_decay=wd, decoupled_wd=True)
+    o.set_state(np.full((1, 2), 8.0, np.float32))
+    for _ in range(T):
+        o.step(np.zeros((1, 2), np.float32), lr)
+    assert np.all(o.w == np.float32(8.0 * (1 - lr * wd) ** T))
+    assert np.all(o.m == 0.0)
+    with pytest.raises(Exception):
+        OracleDaSGD(1, 2, 2, 1, xi=1.0, momentum=0.0, nesterov=True)
+
+
 # ------------------------------------------------------------------ bf16 mode
 
 def test_bf16_rounding_matches_torch_cast():

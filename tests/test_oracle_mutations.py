@@ -15,10 +15,18 @@ SRC = os.path.join(os.path.dirname(oracle.__file__), "dasgd_oracle.cpp")
 
 MUTATIONS = {
     "blend weights swapped": ("xi * wi + one_minus_xi * avg", "one_minus_xi * wi + xi * avg"),
-    "weight decay dropped": ("gi + lambda * static_cast<double>(o->w[i])", "gi"),
+    "weight decay dropped": ("o->decoupled_wd ? gi : gi + lambda * w_old", "gi"),
+    "nesterov looks ahead with the old momentum": (
+        "o->m[i] = static_cast<float>(mu * static_cast<double>(o->m[i]) + gp);\n        dir = o->nesterov ? gp + mu * static_cast<double>(o->m[i])",
+        "const double m_prev = o->m[i];\n        o->m[i] = static_cast<float>(mu * static_cast<double>(o->m[i]) + gp);\n        dir = o->nesterov ? gp + mu * m_prev"),
+    "nesterov ignored": ("dir = o->nesterov ? gp + mu * static_cast<double>(o->m[i]) : static_cast<double>(o->m[i]);",
+                         "dir = static_cast<double>(o->m[i]);"),
+    "decoupled decay also enters the gradient": ("o->decoupled_wd ? gi : gi + lambda * w_old", "gi + lambda * w_old"),
+    "decoupled decay not scaled by the learning rate": ("o->decoupled_wd ? eta * lambda * w_old : 0.0", "o->decoupled_wd ? lambda * w_old : 0.0"),
+    "decoupled decay dropped": ("o->decoupled_wd ? eta * lambda * w_old : 0.0", "0.0"),
     "momentum applied to the sum": ("mu * static_cast<double>(o->m[i]) + gp", "mu * (static_cast<double>(o->m[i]) + gp)"),
-    "step uses the gradient instead of the momentum": ("- eta * static_cast<double>(o->m[i])", "- eta * gp"),
-    "sign of the step": ("static_cast<double>(o->w[i]) - eta * gp", "static_cast<double>(o->w[i]) + eta * gp"),
+    "step uses the gradient instead of the momentum": (": static_cast<double>(o->m[i]);", ": gp;"),
+    "sign of the step": ("w_old - decay - eta * dir", "w_old - decay + eta * dir"),
     "mean not divided": ("acc / static_cast<double>(o->K)", "acc"),
     "mean skips worker 0": ("for (int32_t k = 0; k < o->K; ++k) acc +=", "for (int32_t k = 1; k < o->K; ++k) acc +="),
     "merge fires from the start point": ("d > 0 && u - d >= tau && (u - d) % tau == 0", "d > 0 && (u - d) % tau == 0 && !o->pending.empty()"),
@@ -54,6 +62,10 @@ def battery():
     I.test_delta_merge_keeps_mean_on_plain_sgd()
     I.test_momentum_closed_form_constant_gradient()
     I.test_weight_decay_closed_form_zero_gradient()
+    I.test_nesterov_matches_torch()
+    I.test_decoupled_weight_decay_matches_scaled_weights_then_torch(0.9, False)
+    I.test_decoupled_weight_decay_matches_scaled_weights_then_torch(0.9, True)
+    I.test_decoupled_weight_decay_closed_form_with_momentum()
     I.test_bf16_rounding_matches_torch_cast()
     I.test_bf16_mode_master_equals_f32_run_on_widened_gradients()
     for row in D.table2():
