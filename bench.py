@@ -1,12 +1,16 @@
 #!/usr/bin/env python
 """Benchmark of the DaSGD hot path (local step + snapshot + worker-axis mean + delayed merge).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload resnet50|small]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload resnet50|...]
 
 One "step" is one pass of the whole path over one batch of synthetic gradients: a local step of
 all K replicas, the merge that lands on that step, the snapshot and the side-stream mean.
 Workload "resnet50": K=8 replicas of a P=25.6M float32 vector, momentum 0.9, weight decay 1e-4,
 lr 0.1, tau=1, d=1, xi=0.25.  Prints ONE JSON line (rank 0).
+
+The timed loop of K steps is repeated (--repeats, default 5) and the median is reported, with the
+minimum and maximum beside it.  With --gpus N > 1 and no launcher in the environment the script starts
+its N ranks itself (torch.distributed.run on 127.0.0.1).
 
 --impl reference times the plain CPU checker under oracle/ on the host cores, on a bounded slice of
 the same workload (the path is independent across the parameter index, so a slice is exact).
@@ -16,6 +20,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -42,36 +47,73 @@ WORKLOADS = {
 }
 METRIC = "replica-param updates/s"
 UNIT = "updates/s"
+CHUNK_BYTES = 24 << 20   # target size of one column range of the weight array in the d = 1 pipeline
 
 
 def step_bytes(wl):
-    """Algorithmic HBM bytes per replica-parameter of one local-step launch."""
+    """Algorithmic HBM bytes per replica-parameter of one plain local-step launch."""
     if wl.get("bf16"):
         return (2 + 4 + 4 + 4 + 4 + 2) if wl["momentum"] else (2 + 4 + 4 + 2)
     return 20 if wl["momentum"] else 12   # read w, (m,) g; write w (, m)
 
 
-
-# DRAM traffic of one k_local_step_vec<f32, momentum> launch from an ncu capture on a smaller case
-# (K=8, P=4M; dram__bytes_read.sum + dram__bytes_write.sum = 384.0 + 204.4 MB for 32M updates); it grows
-# in proportion to K*P.  Valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"kernels_sha256_prefix": "329b3ff5ca6ac696", "bytes_per_update": 588.4e6 / 32.0e6,
-               "applies_to": "float32 + momentum"}
+def auto_chunks(K, P):
+    """Column ranges of the d = 1 pipeline by size: ranges of about CHUNK_BYTES of the [K][P] weight array."""
+    return max(2, min(1024, round(K * P * 4 / CHUNK_BYTES)))
 
 
-def profiled_traffic(wl):
-    """Bytes one local-step launch moves through DRAM according to the last ncu capture, or None when
-    the kernels have changed since, or the workload is not the profiled variant."""
+def schedule_of(wl, args):
+    """How bench.py runs dasgd_step for this workload: {'merge': 'chunked'|'fused'|'separate', 'n_chunks', 'lanes'}."""
+    if args.no_fuse:
+        return {"merge": "separate", "n_chunks": 0, "lanes": 0, "copy_snapshot": True}
+    if wl["d"] >= 2:
+        return {"merge": "fused", "n_chunks": 0, "lanes": 0}
+    if wl["d"] == 1 and args.chunks != 1 and wl["P"] >= 2 * 4096:
+        n = args.chunks if args.chunks > 0 else auto_chunks(wl["K"], wl["P"])
+        return {"merge": "chunked", "n_chunks": n, "lanes": 1 if args.lanes else 0}
+    return {"merge": "separate", "n_chunks": 0, "lanes": 0}
+
+
+def path_bytes_per_update(wl, sched):
+    """Algorithmic HBM bytes per replica-parameter update of the whole path as scheduled: tau local
+    steps, the snapshot (0 B with rotating arrays, 8 B as a copy), the mean (4 + 4/K B), and the merge
+    (4/K B when folded into a step kernel, else a pass of its own: 8 + 4/K B, + 2 B for the bfloat16 copy)."""
+    K, tau = wl["K"], wl["tau"]
+    per_cycle = step_bytes(wl) * tau + (4.0 + 4.0 / K)
+    if sched.get("copy_snapshot"):
+        per_cycle += 8.0
+    if sched["merge"] in ("chunked", "fused"):
+        per_cycle += 4.0 / K
+    else:
+        per_cycle += 8.0 + 4.0 / K + (2.0 if wl.get("bf16") else 0.0)
+    return per_cycle / tau
+
+
+# DRAM traffic of the dominant kernel from an ncu capture (profiles/): k_local_step_vec<f32, momentum, xi-merge>
+# on one column range of the pipeline.  Reads grow with the updates of a launch; the stores that are still
+# dirty in L2 when the kernel ends are a constant, not a share.  Valid only while the kernel source is the
+# one that was profiled.
+NCU_TRAFFIC = {"kernels_sha256_prefix": None, "updates": None, "read_bytes": None, "write_bytes": None,
+               "applies_to": "float32 + momentum, merge folded in"}
+
+
+def profiled_traffic(wl, sched, updates_per_launch):
+    """DRAM bytes of one launch of the dominant kernel derived from the last ncu capture, or None when the
+    kernels have changed since or the workload is not the profiled variant."""
     import hashlib
+    if not NCU_TRAFFIC["kernels_sha256_prefix"] or wl.get("bf16") or not wl["momentum"] or sched["merge"] != "chunked":
+        return None
     try:
         src = os.path.join(ROOT, "paper_2006_00441_b200", "csrc", "dasgd_kernels.cuh")
         if hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] != NCU_TRAFFIC["kernels_sha256_prefix"]:
             return None
     except OSError:
         return None
-    if wl.get("bf16") or not wl["momentum"]:
-        return None
-    return NCU_TRAFFIC["bytes_per_update"] * wl["K"] * wl["P"]
+    n0 = NCU_TRAFFIC["updates"]
+    residue = max(0.0, 8.0 * n0 - NCU_TRAFFIC["write_bytes"])          # dirty lines left in L2: constant
+    reads = NCU_TRAFFIC["read_bytes"] * updates_per_launch / n0         # proportional
+    writes = max(0.0, 8.0 * updates_per_launch - residue)
+    return reads + writes
 
 
 def measured_peak_gbs():
@@ -98,7 +140,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", ident, f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50"],
+                ["nvidia-smi", "-i", ident, f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -139,18 +181,18 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ CPU oracle legs
 
-def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmup: int = 0):
+def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmup: int = 0, omp: bool = True):
     """Times the CPU checker on the first P_s parameters of every replica.  Returns a dict."""
     import numpy as np
 
     import oracle
 
     K = wl["K"]
-    probe = oracle.OracleDaSGD(K, 1, 1, 1, 0.5, omp=True)
+    probe = oracle.OracleDaSGD(K, 1, 1, 1, 0.5, omp=omp)
     cores = probe.threads
     probe.close()
     # calibrate on a slice too large for the CPU caches, so the rate is the DRAM-bound one
-    Pc = min(wl["P"], 2_000_000)
+    Pc = min(wl["P"], 2_000_000 if omp else 500_000)
     odt = 1 if wl.get("bf16") else 0
 
     def host_grad(t, idx):
@@ -158,7 +200,7 @@ def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmu
                               dtype=torch.bfloat16 if odt else torch.float32)
         return g.view(torch.int16).numpy().view(np.uint16) if odt else g.numpy()
 
-    o = oracle.OracleDaSGD(K, Pc, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], dtype=odt, omp=True)
+    o = oracle.OracleDaSGD(K, Pc, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], dtype=odt, omp=omp)
     o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=range(Pc)).numpy())
     g = host_grad(0, range(Pc))
     for _ in range(2):
@@ -168,16 +210,17 @@ def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmu
     for _ in range(n_cal):
         o.step(g, wl["lr"])
     rate = K * Pc * n_cal / (time.perf_counter() - t0)  # updates/s, rough
-    o.close()
     if steps is None:       # cpu_baseline leg: fixed slice, as many steps as fit the budget
-        Ps = min(wl["P"], 2_000_000)
+        Ps = Pc
         steps = max(3, min(200, int(seconds_budget * rate / (K * Ps))))
+        ring = [g, host_grad(1, range(Ps))]
     else:                   # reference arm: the caller fixes the steps, the slice is sized to the budget
+        o.close()
         Ps = int(min(wl["P"], 4_000_000, max(1024, seconds_budget * rate / (K * (steps + warmup)))))
-    idx = range(Ps)
-    o = oracle.OracleDaSGD(K, Ps, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], dtype=odt, omp=True)
-    o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=idx).numpy())
-    ring = [host_grad(t, idx) for t in range(2)]
+        idx = range(Ps)
+        o = oracle.OracleDaSGD(K, Ps, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], dtype=odt, omp=omp)
+        o.set_state(inputs.shared_start(0, wl["P"], wl["w_std"], p_index=idx).numpy())
+        ring = [host_grad(t, idx) for t in range(2)]
     for t in range(warmup):
         o.step(ring[t % 2], wl["lr"])
     t0 = time.perf_counter()
@@ -186,10 +229,19 @@ def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmu
     dt = time.perf_counter() - t0
     assert np.isfinite(o.w).all()
     o.close()
+    build = f"OpenMP build of the checker, {cores} threads" if omp else "plain single-thread build of the checker"
     return {"value": K * Ps * steps / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {Ps} of {wl['P']} parameters of all {K} replicas, {steps} steps "
-                      f"(OpenMP build of the checker, {cores} threads)",
+            "sample": f"first {Ps} of {wl['P']} parameters of all {K} replicas, {steps} steps ({build})",
             "seconds": dt, "steps": steps, "P_sample": Ps}
+
+
+def cpu_baseline(wl):
+    """The checker as it stands on the host cores: all cores (OpenMP build) and one thread (plain build)."""
+    par = oracle_throughput(wl, seconds_budget=12.0, omp=True)
+    one = oracle_throughput(wl, seconds_budget=6.0, omp=False)
+    out = {k: par[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    out["single_thread"] = {k: one[k] for k in ("value", "unit", "cores", "sample")}
+    return out
 
 
 def run_reference(args, wl, name):
@@ -202,7 +254,7 @@ def run_reference(args, wl, name):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * r["seconds"] / r["steps"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 gradients, f32 state" if wl.get("bf16") else "f32", "data": "synthetic",
-        "config": workload_config(wl, name),
+        "config": workload_config(wl, name, None),
         "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -210,12 +262,15 @@ def run_reference(args, wl, name):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(wl, name):
-    return {"workload": f"{name}: K={wl['K']} replicas x P={wl['P']} {'bf16 gradients + f32 master' if wl.get('bf16') else 'float32'}, momentum {wl['momentum']}, "
-                        f"weight decay {wl['weight_decay']}, lr {wl['lr']}, tau={wl['tau']}, d={wl['d']}, xi={wl['xi']}",
-            "K": wl["K"], "P": wl["P"], "tau": wl["tau"], "d": wl["d"], "xi": wl["xi"],
-            "l2_policy": "inputs larger than L2 (every step streams all K*P-sized arrays; gradients come from a ring of buffers)",
-            "parallelism": "independent replicas of the workload per GPU (no collective on this path)"}
+def workload_config(wl, name, sched):
+    cfg = {"workload": f"{name}: K={wl['K']} replicas x P={wl['P']} {'bf16 gradients + f32 master' if wl.get('bf16') else 'float32'}, momentum {wl['momentum']}, "
+                       f"weight decay {wl['weight_decay']}, lr {wl['lr']}, tau={wl['tau']}, d={wl['d']}, xi={wl['xi']}",
+           "K": wl["K"], "P": wl["P"], "tau": wl["tau"], "d": wl["d"], "xi": wl["xi"],
+           "l2_policy": "inputs larger than L2 (every step streams all K*P-sized arrays; gradients come from a ring of buffers)",
+           "parallelism": "independent replicas of the workload per GPU (no collective on this path)"}
+    if sched is not None:
+        cfg["schedule"] = sched
+    return cfg
 
 
 # ------------------------------------------------------------------ our arm
@@ -233,133 +288,209 @@ def whole_job(ms_local: float, units_per_rank: float, dist=None, device="cpu"):
     return ms, world * units_per_rank / (ms * 1e-3)
 
 
-def run_ours(args, wl, name):
-    from paper_2006_00441_b200 import binding as B
+class Bench:
+    """One rank's harness: builds contexts for a workload and times loops of steps on them."""
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1 or args.force_dist:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    def __init__(self, args):
+        from paper_2006_00441_b200 import binding as B
+        self.B, self.args = B, args
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+        torch.cuda.set_device(self.local_rank)
+        self.dist = None
+        if self.world > 1 or args.force_dist:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local_rank))
+            self.dist = dist
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
         torch.cuda.synchronize()
 
-    K, P, lr = wl["K"], wl["P"], wl["lr"]
-    bf16 = bool(wl.get("bf16"))
-    gdt = torch.bfloat16 if bf16 else torch.float32
-    RING = wl.get("ring", 4)
-    flags_fused = 0 if args.no_fuse else (B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE)
-    seed = 1000 + rank  # every rank runs its own replica of the workload
+    def flags(self, sched, timing=False):
+        B = self.B
+        if sched["merge"] == "separate" and sched.get("copy_snapshot"):
+            f = 0
+        else:
+            f = B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE
+        if sched.get("lanes"):
+            f |= B.DASGD_FLAG_TWO_LANES
+        return f | (B.DASGD_FLAG_TIMING if timing else 0)
 
-    def make(flags, host_staging=False):
-        e = B.DaSGD(K, P, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"], flags=flags,
-                    dtype=B.DASGD_BF16_MASTER_F32 if bf16 else B.DASGD_F32,
-                    device=local_rank, host_staging=host_staging, order_after_current=False)
-        e.set_state(inputs.shared_start(seed, P, wl["w_std"], device="cuda"))
+    def make(self, wl, sched, timing=False, host_staging=False, flags=None, snapshot_arrays=True):
+        B = self.B
+        e = B.DaSGD(wl["K"], wl["P"], wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"],
+                    flags=self.flags(sched, timing) if flags is None else flags,
+                    dtype=B.DASGD_BF16_MASTER_F32 if wl.get("bf16") else B.DASGD_F32,
+                    n_chunks=sched["n_chunks"] if flags is None else 0, device=self.local_rank,
+                    host_staging=host_staging, order_after_current=False, snapshot_arrays=snapshot_arrays)
+        e.set_state(inputs.shared_start(1000 + self.rank, wl["P"], wl["w_std"], device="cuda"))
         return e
 
-    ring = [inputs.grad_block(seed, t, K, P, wl["g_std"], device="cuda", dtype=gdt) for t in range(RING)]
-    torch.cuda.synchronize()
-
-    def timed_loop(e, steps, warmup, step_fn):
-        for t in range(warmup):
-            step_fn(e, t)
+    def timed(self, e, steps, step_fn, t0=0):
+        """Device time of `steps` calls of step_fn, bracketed by barrier + synchronize; MAX over ranks."""
         e.sync()
-        barrier()
+        self.barrier()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0 = e.launches
         with torch.cuda.stream(e.main):
             ev0.record()
         for t in range(steps):
-            step_fn(e, warmup + t)
+            step_fn(e, t0 + t)
         e.main.wait_stream(e.side)        # the last mean belongs to the timed work
         with torch.cuda.stream(e.main):
             ev1.record()
         e.sync()
-        barrier()
-        ms, _ = whole_job(ev0.elapsed_time(ev1), 0.0, dist, "cuda")
+        self.barrier()
+        ms, _ = whole_job(ev0.elapsed_time(ev1), 0.0, self.dist, "cuda")
         return ms, e.launches - l0
+
+    def repeated(self, e, steps, warmup, repeats, step_fn):
+        """Warm-up, then `repeats` timed loops of exactly `steps` steps.  Returns per-step ms (median, min, max)."""
+        for t in range(warmup):
+            step_fn(e, t)
+        per, launches = [], 0
+        for r in range(repeats):
+            ms, launches = self.timed(e, steps, step_fn, warmup + r * steps)
+            per.append(ms / steps)
+        return {"ms_per_step": statistics.median(per), "min": min(per), "max": max(per), "repeats": repeats,
+                "launches": launches}
+
+
+def measure_workload(bench, wl, sched, steps, warmup, repeats, ring, lr, with_alone=True):
+    """Headline loop + instrumented pass (+ kernels alone) of one workload; returns a dict of figures."""
+    K, P = wl["K"], wl["P"]
+    RING = len(ring)
 
     def dev_step(e, t):
         e.step(ring[t % RING], lr)
 
-    # ---- headline: inputs resident in HBM
-    eng = make(flags_fused)
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    ms, launches = timed_loop(eng, args.steps, args.warmup, dev_step)
-    clocks = sampler.stop() if sampler else None
-    value = world * K * P * args.steps / (ms * 1e-3)
+    out = {}
+    eng = bench.make(wl, sched)
+    out["headline"] = bench.repeated(eng, steps, warmup, repeats, dev_step)
     eng.close()
     del eng
 
-    # ---- instrumented pass: per-kernel device time and the hidden fraction of the averaging
-    eng = make(flags_fused | B.DASGD_FLAG_TIMING)
-    for t in range(args.warmup):
+    # ---- instrumented pass: per-kernel device time and the stalls of the averaging
+    eng = bench.make(wl, sched, timing=True)
+    for t in range(warmup):
         dev_step(eng, t)
     eng.reset_timing()
-    n_inst = min(args.steps, 100)
+    n_inst = min(steps, 100)
     for t in range(n_inst):
-        dev_step(eng, args.warmup + t)
+        dev_step(eng, warmup + t)
     kt = eng.kernel_timing()
-    # the same kernels with nothing else on the GPU (no side-stream mean beside them)
     eng.close()
     del eng
-    eng = make(flags_fused | B.DASGD_FLAG_TIMING)
-    for t in range(3):
-        eng.local_step(ring[t % RING], lr)
-    eng.reset_timing()
-    for t in range(20):
-        eng.local_step(ring[t % RING], lr)
-    eng.sync()
-    for t in range(10):
-        eng.snapshot(); eng.average_async(); eng.sync(); eng.merge(); eng.sync()
-    kt_alone = eng.kernel_timing()
-    eng.close()
-    del eng
-    peak, peak_kind = measured_peak_gbs()
-    n_step, ms_step = kt["local_step"]
-    step_gbs = (K * P * step_bytes(wl) / 1e9) / (ms_step / n_step * 1e-3) if n_step else None
-    alone = {}
-    for kname, nbytes in (("local_step", K * P * step_bytes(wl)), ("mean", K * P * 4 + P * 4),
-                          ("merge", K * P * (10 if bf16 else 8) + P * 4)):
-        n_k, ms_k = kt_alone[kname]
-        if n_k:
-            gbs = nbytes / 1e9 / (ms_k / n_k * 1e-3)
-            alone[kname] = {"ms": ms_k / n_k, "GB/s": gbs, "frac": gbs / peak}
-    # Hidden fraction of the averaging: every microsecond between the two events that bracket the main
-    # stream's wait for a mean counts as stall (that includes the cost of the two events themselves).
-    hidden = None
+    out["kernels_ms_per_launch"] = {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()}
+    out["kernels_ms_per_step"] = {k: v[1] / n_inst for k, v in kt.items()}
+    out["kernel_launches_per_step"] = {k: v[0] / n_inst for k, v in kt.items()}
+    out["instrumented_steps"] = n_inst
     if kt["mean"][0] and kt["mean"][1] > 0:
-        hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
+        out["hidden"] = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
+        out["stall_ms_per_step"] = kt["stall"][1] / n_inst
+    else:
+        out["hidden"] = None
+    if with_alone:
+        # the same kernels with nothing else on the GPU (no side-stream mean beside them)
+        plain = dict(sched, merge="separate", n_chunks=0, lanes=0)
+        eng = bench.make(wl, plain, timing=True)
+        for t in range(3):
+            eng.local_step(ring[t % RING], lr)
+        eng.reset_timing()
+        for t in range(20):
+            eng.local_step(ring[t % RING], lr)
+        eng.sync()
+        for t in range(10):
+            eng.snapshot(); eng.average_async(); eng.sync(); eng.merge(); eng.sync()
+        kt_alone = eng.kernel_timing()
+        eng.close()
+        del eng
+        peak, _ = measured_peak_gbs()
+        alone = {}
+        bf16 = bool(wl.get("bf16"))
+        for kname, nbytes in (("local_step", K * P * step_bytes(wl)), ("mean", K * P * 4 + P * 4),
+                              ("merge", K * P * (10 if bf16 else 8) + P * 4)):
+            n_k, ms_k = kt_alone[kname]
+            if n_k:
+                gbs = nbytes / 1e9 / (ms_k / n_k * 1e-3)
+                alone[kname] = {"ms": ms_k / n_k, "GB/s": gbs, "frac": gbs / peak}
+        out["alone"] = alone
+    return out
 
-    hidden_cost = None
-    if all(k in alone for k in ("local_step", "mean", "merge")):
-        tau_, d_ = wl["tau"], wl["d"]
-        main_alone = tau_ * alone["local_step"]["ms"] + (alone["merge"]["ms"] if d_ < 2 else 0.0)
-        hidden_cost = 1.0 - (ms / args.steps * tau_ - main_alone) / alone["mean"]["ms"]
+
+def hidden_cost(wl, sched, ms_per_step, alone):
+    """1 - (cycle time - cycle time of the main-stream kernels alone) / mean kernel alone."""
+    if not all(k in alone for k in ("local_step", "mean", "merge")):
+        return None
+    tau, K = wl["tau"], wl["K"]
+    main_alone = tau * alone["local_step"]["ms"]
+    if sched["merge"] == "separate":
+        main_alone += alone["merge"]["ms"]
+    else:   # folded in: the step kernel that merges also reads the mean once per row
+        main_alone += alone["local_step"]["ms"] * (4.0 / K) / step_bytes(wl)
+    return 1.0 - (ms_per_step * tau - main_alone) / alone["mean"]["ms"]
+
+
+def run_ours(args, wl, name, bench=None, compact=False):
+    bench = bench or Bench(args)
+    B, rank, world = bench.B, bench.rank, bench.world
+    K, P, lr = wl["K"], wl["P"], wl["lr"]
+    bf16 = bool(wl.get("bf16"))
+    gdt = torch.bfloat16 if bf16 else torch.float32
+    RING = wl.get("ring", 4)
+    sched = schedule_of(wl, args)
+    seed = 1000 + rank  # every rank runs its own replica of the workload
+    ring = [inputs.grad_block(seed, t, K, P, wl["g_std"], device="cuda", dtype=gdt) for t in range(RING)]
+    torch.cuda.synchronize()
+
+    def dev_step(e, t):
+        e.step(ring[t % RING], lr)
+
+    sampler = ClockSampler(bench.local_rank) if rank == 0 and not compact else None
+    m = measure_workload(bench, wl, sched, args.steps, args.warmup, args.repeats, ring, lr,
+                         with_alone=(not compact) or args.sweep)
+    clocks = sampler.stop() if sampler else None
+    ms = m["headline"]["ms_per_step"]
+    value = world * K * P / (ms * 1e-3)
+    bpu = path_bytes_per_update(wl, sched)
+    if compact:
+        del ring
+        torch.cuda.empty_cache()
+        return {"value": value, "unit": UNIT, "ms_per_step": ms, "ms_min": m["headline"]["min"], "ms_max": m["headline"]["max"],
+                "repeats": args.repeats, "steps": args.steps, "gpu_launches_per_step": m["headline"]["launches"] / args.steps,
+                "schedule": sched, "bytes_per_update": bpu, "whole_path_gbs": value / world * bpu / 1e9,
+                "averaging_hidden_frac": m["hidden"], "kernels_ms_per_step": m["kernels_ms_per_step"],
+                "alone": m.get("alone")}
+
+    peak, peak_kind = measured_peak_gbs()
+    alone = m["alone"]
+    # The dominant kernel is the local step (with the merge folded in under the chunked / fused schedules).
+    # Its launches tile the main stream's whole iteration, so its live rate is taken over the timed region
+    # itself: algorithmic bytes of one iteration's step launches / median time of one iteration.  Boundaries
+    # between launches and the bandwidth the side-stream mean takes all count against it.
+    launches_step = m["kernel_launches_per_step"]["local_step"]
+    merge_in_step = sched["merge"] in ("chunked", "fused")
+    step_b = step_bytes(wl) + ((4.0 / K) / wl["tau"] if merge_in_step else 0.0)
+    main_ms = ms if merge_in_step else ms - (m["kernels_ms_per_step"]["merge"] or 0.0)
+    step_gbs = K * P * step_b / 1e9 / (main_ms * 1e-3)
+    updates_per_launch = K * P / launches_step if launches_step else K * P
 
     # ---- ablation: the same work with the mean computed inside the step kernel (no side stream)
     ablation = None
     if not args.no_ablation:
-        eng = B.DaSGD(K, P, wl["tau"], wl["d"], wl["xi"], wl["momentum"], wl["weight_decay"],
-                      flags=B.DASGD_FLAG_INLINE_MEAN, dtype=B.DASGD_BF16_MASTER_F32 if bf16 else B.DASGD_F32,
-                      device=local_rank, order_after_current=False, snapshot_arrays=False)
-        eng.set_state(inputs.shared_start(seed, P, wl["w_std"], device="cuda"))
-        ms_a, launches_a = timed_loop(eng, args.steps, args.warmup, dev_step)
+        eng = bench.make(wl, sched, flags=B.DASGD_FLAG_INLINE_MEAN, snapshot_arrays=False)
+        a = bench.repeated(eng, args.steps, args.warmup, min(3, args.repeats), dev_step)
         bytes_a = (step_bytes(wl) * wl["tau"] + 8.0 / K) / wl["tau"]
         ablation = {"schedule": "inline mean: one kernel per iteration, mean summed in registers, no snapshot, "
                                 "no side stream (same results; the averaging is no longer asynchronous)",
-                    "value": world * K * P * args.steps / (ms_a * 1e-3), "unit": UNIT, "ms_per_step": ms_a / args.steps,
-                    "gpu_launches": launches_a, "bytes_per_update": bytes_a,
-                    "whole_path_gbs": K * P * args.steps / (ms_a * 1e-3) * bytes_a / 1e9}
+                    "value": world * K * P / (a["ms_per_step"] * 1e-3), "unit": UNIT, "ms_per_step": a["ms_per_step"],
+                    "gpu_launches": a["launches"], "bytes_per_update": bytes_a,
+                    "whole_path_gbs": K * P / (a["ms_per_step"] * 1e-3) * bytes_a / 1e9}
         eng.close()
         del eng
 
@@ -368,7 +499,7 @@ def run_ours(args, wl, name):
     try:
         if args.no_e2e:
             raise RuntimeError("skipped (--no-e2e)")
-        eng = make(flags_fused, host_staging=2)
+        eng = bench.make(wl, sched, host_staging=2)
         hosts = [torch.empty((K, P), dtype=gdt).pin_memory() for _ in range(2)]
         for i, h in enumerate(hosts):
             h.copy_(ring[i])
@@ -379,94 +510,147 @@ def run_ours(args, wl, name):
         def host_step(e, t):
             e.step_host(hosts[t % 2], lr, probe)
 
-        ms_e, _ = timed_loop(eng, e2e_steps, 3, host_step)
-        e2e = {"value": world * K * P * e2e_steps / (ms_e * 1e-3), "unit": UNIT,
+        h = bench.repeated(eng, e2e_steps, 3, min(3, args.repeats), host_step)
+        e2e = {"value": world * K * P / (h["ms_per_step"] * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": K * P * (2 if bf16 else 4), "d2h_bytes_per_step": probe.numel() * 4,
-               "steps": e2e_steps, "ms_per_step": ms_e / e2e_steps}
+               "steps": e2e_steps, "ms_per_step": h["ms_per_step"], "ms_min": h["min"], "ms_max": h["max"],
+               "repeats": h["repeats"]}
         eng.close()
         del eng, hosts
     except Exception as ex:  # page-locked memory can be refused on a small host
         e2e = {"value": None, "unit": UNIT, "error": str(ex)[:200]}
 
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
     del ring
     torch.cuda.empty_cache()
+    others = None
+    if rank == 0 and world == 1 and not args.no_others:
+        others = other_workloads(args, bench)
+    if bench.dist is not None:
+        bench.dist.barrier()
+        bench.dist.destroy_process_group()
     if rank != 0:
         return None
 
-    cpu = (oracle_throughput(wl, seconds_budget=15.0) if not args.no_cpu else
+    cpu = (cpu_baseline(wl) if not args.no_cpu else
            {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": "skipped (--no-cpu)"})
+    kname = "k_local_step_vec (%s%s%s)" % ("bf16 gradients + f32 master" if bf16 else "float32",
+                                           ", momentum" if wl["momentum"] else "", ", xi-merge folded in" if merge_in_step else "")
+    stall = m.get("stall_ms_per_step")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 gradients, f32 state" if bf16 else "f32", "data": "synthetic", "config": workload_config(wl, name),
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "k_local_step_vec (%s%s)" % ("bf16 gradients + f32 master" if bf16 else "float32",
-                                                                ", momentum" if wl["momentum"] else ""),
+        "ms_per_step": ms, "ms_per_step_min": m["headline"]["min"], "ms_per_step_max": m["headline"]["max"],
+        "repeats": args.repeats, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 gradients, f32 state" if bf16 else "f32", "data": "synthetic",
+        "config": workload_config(wl, name, sched),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": m["headline"]["launches"],
+        "roofline": {"bound": "hbm", "kernel": kname,
                      "achieved": step_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": (step_gbs / peak) if step_gbs else None, "peak_kind": f"of {peak_kind}",
-                     "frac_of_8TBs": (step_gbs / 8000.0) if step_gbs else None,
-                     "algorithmic_bytes_per_launch": K * P * step_bytes(wl),
-                     "avg_launch_ms": (ms_step / n_step) if n_step else None,
-                     "timed": f"CUDA events on the launching stream, instrumented pass of {n_inst} steps; the "
-                              "side-stream mean kernel runs beside this kernel and shares HBM with it",
-                     "traffic": profiled_traffic(wl),
-                     "traffic_note": "ncu dram bytes of a K=8, P=4M launch scaled by K*P; below the algorithmic "
-                                     "bytes because the last stores are still dirty in L2 when the kernel ends",
+                     "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_8TBs": step_gbs / 8000.0,
+                     "algorithmic_bytes_per_update": step_b,
+                     "algorithmic_bytes_per_launch": updates_per_launch * step_b,
+                     "launches_per_step": launches_step,
+                     "avg_launch_ms": main_ms / launches_step if launches_step else None,
+                     "timed": "over the timed region: the kernel's launches tile the main stream's iteration, so the "
+                              "average launch time is the median iteration time / launches per iteration (launch "
+                              "boundaries and the bandwidth taken by the side-stream mean count against the kernel)",
+                     "instrumented_ms_per_launch": m["kernels_ms_per_launch"]["local_step"],
+                     "instrumented_note": "CUDA events around each launch in a separate pass; with two lanes consecutive "
+                                          "launches overlap, so these do not add up to the iteration time",
+                     "traffic": profiled_traffic(wl, sched, updates_per_launch),
+                     "traffic_note": "ncu dram bytes of one launch of the same shape (reads scale with the updates of a "
+                                     "launch; the stores still dirty in L2 at kernel end are a constant); null when the "
+                                     "kernels changed since the capture",
                      "alone": alone},
-        "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
-        "averaging_hidden_frac": hidden,
-        "averaging_hidden_frac_cost": hidden_cost,
-        "averaging_hidden_note": "averaging_hidden_frac: share of the mean kernel's time during which the main stream "
-                                 "did not wait for it (the paper's notion: the critical path never stalls).  "
-                                 "_cost: 1 - (cycle time - cycle time of the main-stream kernels alone) / mean kernel "
-                                 "alone; on one GPU the mean competes with the local step for the same HBM, so its "
-                                 "bytes are not free even though nothing waits for it",
-        "whole_path_gbs": value / world * path_bytes_per_update(wl) / 1e9,
+        "kernels_ms_per_launch": m["kernels_ms_per_launch"],
+        "kernels_ms_per_step": m["kernels_ms_per_step"],
+        "averaging_hidden_frac": m["hidden"],
+        "averaging_stall_ms_per_step": stall,
+        "averaging_hidden_frac_vs_mean_alone": (1.0 - stall * wl["tau"] / alone["mean"]["ms"])
+        if stall is not None and "mean" in alone else None,
+        "averaging_hidden_frac_cost": hidden_cost(wl, sched, ms, alone),
+        "averaging_hidden_note": "averaging_hidden_frac = 1 - (time streams were blocked waiting for a mean) / (time the mean "
+                                 "kernels ran), the paper's notion: the critical path does not stall; a wait's stall is "
+                                 "[mean complete] - [waiting stream idle], from CUDA events, when positive.  _vs_mean_alone "
+                                 "divides by the mean's time on an idle GPU instead.  _cost = 1 - (cycle time - cycle time "
+                                 "of the main-stream kernels alone) / mean kernel alone: on one GPU the mean draws on the "
+                                 "same HBM as the local step, so its bytes are not free even though nothing waits for it",
+        "bytes_per_update": bpu,
+        "whole_path_gbs": value / world * bpu / 1e9,
+        "whole_path_frac_of_measured": value / world * bpu / 1e9 / peak,
         "ablation_inline_mean": ablation,
-        "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "other_workloads": others,
+        "cpu_baseline": cpu,
     }
     return line
 
 
+def other_workloads(args, bench):
+    """Compact figures for the other configurations (each a short run): the linear-regression size, the
+    bfloat16 BERT-large size, two corners of the K x tau x d sweep, and the MLP workload."""
+    import copy
+    a = copy.copy(args)
+    a.warmup, a.repeats, a.sweep = 3, 3, False
+    out = {}
+    t0 = time.perf_counter()
+    for key, wl, steps in (("small_K4_P1024_tau4_d1", dict(WORKLOADS["small"], ring=2), 200),
+                           ("sweep_K2_tau1_d1", dict(WORKLOADS["resnet50"], K=2, weight_decay=0.0, ring=2), 20),
+                           ("sweep_K32_tau4_d2", dict(WORKLOADS["resnet50"], K=32, tau=4, d=2, weight_decay=0.0, ring=1), 20),
+                           ("bert_large_bf16_K4_P335M_tau2_d1", dict(WORKLOADS["bert_large"], ring=1), 20)):
+        try:
+            a.steps = steps
+            out[key] = run_ours(a, wl, key, bench=bench, compact=True)
+            out[key].pop("alone", None)
+        except Exception as ex:
+            out[key] = {"error": str(ex)[:200]}
+        torch.cuda.empty_cache()
+    try:
+        a.steps, a.warmup = 30, 3
+        out["mlp_K8_4x4096_tau1_d1"] = mlp_figures(a)
+    except Exception as ex:
+        out["mlp_K8_4x4096_tau1_d1"] = {"error": str(ex)[:200]}
+    torch.cuda.empty_cache()
+    out["seconds"] = time.perf_counter() - t0
+    return out
+
+
 def run_sweep(args):
-    """The K x tau x d sweep at P = 25.6M float32 (one JSON line per point), then the bf16 workload."""
-    args.no_e2e = args.no_cpu = True
+    """The K x tau x d sweep at P = 25.6M float32 (one JSON line per point)."""
+    args.no_e2e = args.no_cpu = args.no_others = True
+    bench = Bench(args)
     for K in (2, 4, 8, 16, 32):
         for tau in (1, 2, 4):
             for d in (1, 2):
-                wl = dict(WORKLOADS["resnet50"], K=K, tau=tau, d=d, weight_decay=0.0)
-                line = run_ours(args, wl, "sweep")
-                if line:
-                    keep = {k: line[k] for k in ("value", "ms_per_step", "gpu_launches", "averaging_hidden_frac",
-                                                 "whole_path_gbs", "kernels_ms_per_launch")}
-                    if line.get("ablation_inline_mean"):
-                        keep["inline_mean_value"] = line["ablation_inline_mean"]["value"]
-                        keep["inline_mean_gbs"] = line["ablation_inline_mean"]["whole_path_gbs"]
-                    keep.update(K=K, tau=tau, d=d, local_step_alone_gbs=line["roofline"]["alone"]["local_step"]["GB/s"])
-                    print(json.dumps(keep), flush=True)
+                wl = dict(WORKLOADS["resnet50"], K=K, tau=tau, d=d, weight_decay=0.0, ring=2 if K >= 16 else 4)
+                r = run_ours(args, wl, "sweep", bench=bench, compact=True)
+                r.update(K=K, tau=tau, d=d)
+                if r.get("alone"):
+                    r["local_step_alone_gbs"] = r["alone"]["local_step"]["GB/s"]
+                    r["mean_alone_gbs"] = r["alone"]["mean"]["GB/s"]
+                r.pop("alone", None)
+                print(json.dumps(r), flush=True)
 
 
-def run_mlp(args):
+def mlp_figures(args):
     """End-to-end workload: K=8 replicas of a 4-layer, 4096-wide bf16 MLP trained against a fixed random
     teacher (batch 256 per worker; forward/backward = batched bf16 matmuls of the GEMM library, on the
     main stream), DaSGD update path with tau=1, d=1.  Here the averaging overlaps real compute."""
     from paper_2006_00441_b200 import binding as B
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
     K, H, L, batch, lr, tau, d, xi = 8, 4096, 4, 256, 1e-3, 1, 1, 0.25
     net = inputs.TeacherMLP(4, K, H, layers=L, batch=batch, device="cuda", dtype=torch.bfloat16)
     net.precompute_batches(4)
     P = net.P
     flops_per_step = 3 * 2 * K * batch * H * H * L      # forward + two backward GEMMs per layer
-    out = {}
-    for name, flags in (("async", B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE | B.DASGD_FLAG_TIMING),
-                        ("inline_mean", B.DASGD_FLAG_INLINE_MEAN | B.DASGD_FLAG_TIMING)):
+    base = B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE | B.DASGD_FLAG_TIMING
+    n_chunks = auto_chunks(K, P)
+    variants = (("separate_merge", base, 0), ("merge_in_step_kernel", base | B.DASGD_FLAG_FUSE_MERGE_D1, 0),
+                ("chunked_pipeline", base | B.DASGD_FLAG_TWO_LANES, n_chunks),
+                ("inline_mean", B.DASGD_FLAG_INLINE_MEAN | B.DASGD_FLAG_TIMING, 0))
+    out = {"P": P, "n_chunks": n_chunks}
+    for name, flags, chunks in variants:
         e = B.DaSGD(K, P, tau, d, xi, 0.9, 0.0, dtype=B.DASGD_BF16_MASTER_F32, flags=flags, order_after_current=False,
-                    snapshot_arrays=(name == "async"))
+                    snapshot_arrays=(name != "inline_mean"), n_chunks=chunks)
         e.set_state(net.student_init())
         g = torch.zeros(K, P, dtype=torch.bfloat16, device="cuda")
         torch.cuda.synchronize()
@@ -491,44 +675,53 @@ def run_mlp(args):
             ev[1].record()
             # forward/backward alone, for the breakdown
             e.sync()
-            for t in range(20):
+            for t in range(10):
                 net.forward_backward(t, e.w_lp, g)
             ev[2].record()
         e.sync()
         torch.cuda.synchronize()
         ms = ev[0].elapsed_time(ev[1]) / args.steps
-        ms_fb = ev[1].elapsed_time(ev[2]) / 20
+        ms_fb = ev[1].elapsed_time(ev[2]) / 10
         kt = e.kernel_timing()
         hidden = None
         if kt["mean"][0] and kt["mean"][1] > 0:
             hidden = max(0.0, 1.0 - kt["stall"][1] / kt["mean"][1])
-        out[name] = {"value": K * P * args.steps / (ms * args.steps * 1e-3), "ms_per_step": ms,
+        out[name] = {"value": K * P / (ms * 1e-3), "ms_per_step": ms,
                      "ms_forward_backward": ms_fb, "gemm_tflops": flops_per_step / (ms_fb * 1e-3) / 1e12,
-                     "ms_update_path": ms - ms_fb, "gpu_launches": e.launches - l0, "averaging_hidden_frac": hidden,
-                     "kernels_ms_per_launch": {k: (v[1] / v[0] if v[0] else None) for k, v in kt.items()},
+                     "ms_update_path": ms - ms_fb, "gpu_launches_per_step": (e.launches - l0) / args.steps,
+                     "averaging_hidden_frac": hidden,
+                     "kernels_ms_per_step": {k: v[1] / args.steps for k, v in kt.items()},
                      "loss_first_last": [float(x.mean()) for x in losses]}
         e.close()
         del e, g
         torch.cuda.empty_cache()
-    line = {"metric": METRIC, "value": out["async"]["value"], "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": out["async"]["ms_per_step"], "higher_is_better": True,
+    # cost-based figure: what the asynchronous mean adds to the update path beyond the main-stream kernels
+    for name in ("separate_merge", "merge_in_step_kernel", "chunked_pipeline"):
+        k = out[name]["kernels_ms_per_step"]
+        if k["mean"] > 0 and name != "chunked_pipeline":   # two lanes: the per-launch times overlap, no such sum
+            out[name]["averaging_hidden_frac_cost"] = 1.0 - (out[name]["ms_update_path"] - k["local_step"] - k["merge"]) / k["mean"]
+    return out
+
+
+def run_mlp(args):
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    r = mlp_figures(args)
+    best = min((r[k] for k in ("separate_merge", "merge_in_step_kernel", "chunked_pipeline")), key=lambda x: x["ms_per_step"])
+    line = {"metric": METRIC, "value": best["value"], "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": best["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/gradients/activations, f32 master", "data": "synthetic",
-            "config": {"workload": f"mlp: K={K} replicas of a {L}-layer {H}-wide bias-free ReLU MLP (P={P}), batch {batch} per "
-                                   f"worker, teacher-student regression, momentum 0.9, lr {lr}, tau={tau}, d={d}, xi={xi}",
-                       "K": K, "P": P, "tau": tau, "d": d, "xi": xi},
-            "async": out["async"], "inline_mean": out["inline_mean"]}
+            "config": {"workload": f"mlp: K=8 replicas of a 4-layer 4096-wide bias-free ReLU MLP (P={r['P']}), batch 256 per "
+                                   f"worker, teacher-student regression, momentum 0.9, lr 0.001, tau=1, d=1, xi=0.25",
+                       "K": 8, "P": r["P"], "tau": 1, "d": 1, "xi": 0.25}}
+    line.update(r)
     print(json.dumps(line), flush=True)
 
 
-def path_bytes_per_update(wl):
-    """Algorithmic HBM bytes per replica-parameter update of the whole path as bench.py schedules it
-    (rotating snapshots, merge folded into a step kernel when d >= 2): tau local steps, the snapshot
-    (0 B: no copy), the mean (4 + 4/K B), and the merge (4/K B inside a step kernel when d >= 2, else a
-    pass of its own: 8 + 4/K B, + 2 B for the bfloat16 copy)."""
-    K, tau, d = wl["K"], wl["tau"], wl["d"]
-    per_cycle = step_bytes(wl) * tau + (4.0 + 4.0 / K)
-    per_cycle += (4.0 / K) if d >= 2 else (8.0 + 4.0 / K + (2.0 if wl.get("bf16") else 0.0))
-    return per_cycle / tau
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
 
 
 def main():
@@ -536,6 +729,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=5, help="timed loops of --steps steps; the median is reported")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS) + ["mlp"])
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (profiling on a small case)")
@@ -544,14 +738,24 @@ def main():
     ap.add_argument("--d", type=int, default=-1, help="override the delay (sweep)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--no-fuse", action="store_true", help="run the unfused schedule (separate snapshot copy and merge)")
     ap.add_argument("--force-dist", action="store_true",
                     help="initialise the NCCL process group even with one rank (exercises the multi-rank plumbing)")
     ap.add_argument("--no-ablation", action="store_true", help="skip the inline-mean ablation leg")
+    ap.add_argument("--lanes", type=int, default=1, help="1: alternate the column ranges between two streams; 0: one stream")
+    ap.add_argument("--chunks", type=int, default=0,
+                    help="column ranges of the d = 1 pipeline (merge folded into the step kernel); 0: by size "
+                         "(ranges of about 24 MiB of weights); 1: off (separate merge kernel)")
     ap.add_argument("--sweep", action="store_true", help="run the K x tau x d sweep instead (one JSON line per point)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus > 1 and "RANK" not in os.environ and args.impl == "ours":
+        # no launcher in the environment: start the ranks here, one per GPU, on the loopback address
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     wl = dict(WORKLOADS.get(args.workload, {}))
     if args.P > 0:
         wl["P"] = args.P

@@ -61,8 +61,10 @@ typedef enum {
 #define DASGD_FLAG_TIMING 0x1u        /* record CUDA events around every average and every wait for it */
 #define DASGD_FLAG_FUSE_SNAPSHOT 0x2u /* dasgd_step: store the snapshot from the kernel that last writes
                                          w in that step instead of running a separate copy             */
-#define DASGD_FLAG_FUSE_MERGE 0x4u    /* dasgd_step: when d >= 2, blend the mean inside the local-step
-                                         kernel of the step the merge lands on                         */
+#define DASGD_FLAG_FUSE_MERGE 0x4u    /* dasgd_step: blend the mean inside the local-step kernel of the step
+                                         the merge lands on (Eq. 2's second branch as one assignment).
+                                         Applies when d >= 2, and when d == 1 if n_chunks > 1 or
+                                         DASGD_FLAG_FUSE_MERGE_D1 is set                                */
 
 #define DASGD_FLAG_ROTATE_SNAPSHOT 0x8u /* snapshots cost no copy: w and the n_slots arrays of snap form a
                                          pool of n_slots+1 weight arrays; a snapshot freezes the array that
@@ -79,8 +81,22 @@ typedef enum {
                                          mean is no longer computed asynchronously.  xi-blend merge only.  The
                                          explicit snapshot/average/merge calls keep working if snap is given. */
 
-/* Variants of the local step.  The paper names only "weight decay 0.01, moment 0.9" on its platform
- * (Section IV-A) and gives no formula, so the common forms are all offered; the default is the plain one. */
+#define DASGD_FLAG_FUSE_MERGE_D1 0x80u /* with DASGD_FLAG_FUSE_MERGE and n_chunks <= 1: fold the merge into the
+                                         step kernel also when d == 1.  The kernel of step s+1 then cannot start
+                                         before the mean of step s is complete, so this pays off only when the
+                                         caller's own work between two steps (forward/backward) gives the mean
+                                         its window (the condition t_c < d*t_p of Eq. 6); with back-to-back steps
+                                         use n_chunks instead                                                   */
+
+#define DASGD_FLAG_TWO_LANES 0x100u    /* with n_chunks > 1: the step kernels of odd column ranges run on a second
+                                         stream owned by the library, forked from the main stream at the start of
+                                         the dasgd_step call and joined to it at its end, so that consecutive
+                                         ranges overlap at their boundaries.  Work the caller enqueues on the
+                                         main stream before / after the call is still ordered before / after all
+                                         of it.  Results are unchanged.                                        */
+
+/* Variants of the local step.  Section IV-A states only the values of momentum and weight decay used on the
+ * paper's platform and gives no formula, so the common forms are all offered; the default is the plain one. */
 #define DASGD_FLAG_NESTEROV 0x20u      /* w <- w - lr*(g' + mu*m) with the freshly updated m (needs momentum > 0) */
 #define DASGD_FLAG_DECOUPLED_WD 0x40u  /* g' = g, and w <- w - lr*lambda*w - lr*(step direction): the decay acts
                                           on the weights directly instead of entering the momentum            */
@@ -103,7 +119,13 @@ typedef struct dasgd_config {
   uint32_t sync_timeout_ms; /* dasgd_sync gives up after this long; 0 means 60000                     */
   int32_t n_stage;      /* gradient staging arrays behind g_stage: 0 (none), 1, or 2 (the copy of the
                            next step's gradients then overlaps this step's kernels)                   */
-  int32_t reserved;     /* set to 0                                                                   */
+  int32_t n_chunks;     /* 0 or 1: off.  C > 1 (at most 1024; needs d >= 1, DASGD_FLAG_ROTATE_SNAPSHOT and
+                           DASGD_FLAG_FUSE_MERGE): when d == 1, dasgd_step cuts the parameter axis into C
+                           column ranges and pipelines them: the step kernel of range c (which blends the
+                           mean of range c that lands) is followed on the side stream by the mean of range
+                           c of the new snapshot, which runs beside the step kernels of ranges c+1, ...
+                           The merge then costs no pass of its own although the mean of step s is consumed
+                           by step s+1.  Results are the same as without chunks.                        */
   void *w;              /* device, [K][ld] float32, in/out: weights (master weights in bf16 mode); with
                            DASGD_FLAG_ROTATE_SNAPSHOT: where the weights START (see dasgd_get_weights)  */
   void *m;              /* device, [K][ld] float32, in/out: momentum buffers (start them at 0)        */
@@ -167,20 +189,24 @@ dasgd_status dasgd_get_weights(const dasgd_ctx *ctx, void **w_device);
 /* t, the number of completed local steps, and the number of snapshots awaiting their merge. */
 dasgd_status dasgd_get_step(const dasgd_ctx *ctx, int64_t *t, int32_t *pending);
 
-/* Device pointers of the i-th oldest pending slot (0 = oldest) and the step it was taken at. */
+/* Device pointers of the i-th oldest pending slot (0 = oldest) and the step it was taken at.
+ * *snap_device is NULL for a slot made by the DASGD_FLAG_INLINE_MEAN schedule (it has a mean but no
+ * snapshot array). */
 dasgd_status dasgd_get_pending(const dasgd_ctx *ctx, int32_t i, int64_t *s, void **snap_device,
                                void **mean_device);
 
 /* Requires DASGD_FLAG_TIMING.  Synchronises, then returns sums over all averages completed since
- * the last dasgd_reset_timing: n_avg averages, ms_avg = time the averaging kernels took on the side stream,
- * ms_stall = time the main stream spent waiting for them before merges.  The fraction of
+ * the last dasgd_reset_timing: n_avg mean launches, ms_avg = time the mean kernels took on the side stream,
+ * ms_stall = time streams spent blocked on them.  The stall of one wait is measured between two CUDA events
+ * on the device clock: "the waiting stream has finished everything queued before the wait" and "the mean
+ * kernel is complete"; it counts when the second comes after the first, else it is 0.  The fraction of
  * averaging hidden behind local work is 1 - ms_stall/ms_avg (Section V, Eq. 6). */
 dasgd_status dasgd_get_timing(dasgd_ctx *ctx, int64_t *n_avg, double *ms_avg, double *ms_stall);
 
 /* Requires DASGD_FLAG_TIMING.  Synchronises, then returns the number of launches and the summed
  * device time (CUDA events on the launching stream) of one kind of work since the last
  * dasgd_reset_timing: which = 0 local-step kernels (fused variants included), 1 snapshot copies,
- * 2 worker-axis means, 3 merge kernels, 4 the main stream's waits for a mean. */
+ * 2 worker-axis means, 3 merge kernels, 4 the waits for a mean (n = waits issued, ms = time blocked). */
 dasgd_status dasgd_get_kernel_timing(dasgd_ctx *ctx, int32_t which, int64_t *n, double *ms);
 
 /* Synchronises and zeroes every timing counter. */
@@ -209,6 +235,17 @@ dasgd_status dasgd_delay_guideline(double t_c, double t_p, int32_t *d, int32_t *
  * times in milliseconds. */
 dasgd_status dasgd_advise_delay(dasgd_ctx *ctx, double extra_tp_ms, int32_t *d, int32_t *tau, double *t_c_ms,
                                 double *t_p_ms);
+
+/* Requires DASGD_FLAG_TIMING.  Synchronises, then returns how many replica-parameters (K times the columns
+ * of each launch) the timed launches of one kind have processed since the last dasgd_reset_timing; `which`
+ * as in dasgd_get_kernel_timing (4, the waits, always gives 0).  With n_chunks > 1 one step is several
+ * launches, so bytes per second follow from units and time, not from the launch count. */
+dasgd_status dasgd_get_kernel_units(dasgd_ctx *ctx, int32_t which, int64_t *units);
+
+/* bf16 mode: rewrites the bfloat16 copy w_lp from the float32 master weights (round to nearest even) with
+ * the library's own conversion, on the main stream.  Call it after writing initial weights into w, so that
+ * no rounding of the method's state happens outside the library.  DASGD_ERR_BAD_STATE in float32 mode. */
+dasgd_status dasgd_refresh_lp(dasgd_ctx *ctx);
 
 /* Number of kernels this context has launched so far. */
 dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches);

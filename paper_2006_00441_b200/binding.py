@@ -26,12 +26,15 @@ DASGD_MERGE_XI, DASGD_MERGE_DELTA = 0, 1
 DASGD_FLAG_TIMING, DASGD_FLAG_FUSE_SNAPSHOT, DASGD_FLAG_FUSE_MERGE, DASGD_FLAG_ROTATE_SNAPSHOT = 0x1, 0x2, 0x4, 0x8
 DASGD_FLAG_INLINE_MEAN = 0x10
 DASGD_FLAG_NESTEROV, DASGD_FLAG_DECOUPLED_WD = 0x20, 0x40
+DASGD_FLAG_FUSE_MERGE_D1 = 0x80
+DASGD_FLAG_TWO_LANES = 0x100
 
 EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",
     "dasgd_step", "dasgd_step_host", "dasgd_get_weights", "dasgd_get_step", "dasgd_get_pending", "dasgd_get_timing",
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
     "dasgd_average_merge_noalloc", "dasgd_delay_guideline", "dasgd_advise_delay", "dasgd_export_state", "dasgd_import_state",
+    "dasgd_get_kernel_units", "dasgd_refresh_lp",
 ]
 
 
@@ -41,7 +44,7 @@ class dasgd_config(ctypes.Structure):
         ("merge_mode", ctypes.c_int32), ("n_slots", ctypes.c_int32), ("flags", ctypes.c_uint32),
         ("device", ctypes.c_int32), ("P", ctypes.c_int64), ("ld", ctypes.c_int64),
         ("xi", ctypes.c_float), ("momentum", ctypes.c_float), ("weight_decay", ctypes.c_float),
-        ("sync_timeout_ms", ctypes.c_uint32), ("n_stage", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("sync_timeout_ms", ctypes.c_uint32), ("n_stage", ctypes.c_int32), ("n_chunks", ctypes.c_int32),
         ("w", ctypes.c_void_p), ("m", ctypes.c_void_p), ("w_lp", ctypes.c_void_p), ("snap", ctypes.c_void_p),
         ("mean", ctypes.c_void_p), ("g_stage", ctypes.c_void_p),
         ("main_stream", ctypes.c_void_p), ("side_stream", ctypes.c_void_p),
@@ -75,6 +78,8 @@ def _load() -> ctypes.CDLL:
                                    ctypes.POINTER(ctypes.c_double)]
     L.dasgd_get_launches.argtypes = [vp, ctypes.POINTER(i64)]
     L.dasgd_get_kernel_timing.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.dasgd_get_kernel_units.argtypes = [vp, i32, ctypes.POINTER(i64)]
+    L.dasgd_refresh_lp.argtypes = [vp]
     L.dasgd_reset_timing.argtypes = [vp]
     L.dasgd_strerror.argtypes = [ctypes.c_int]
     L.dasgd_strerror.restype = ctypes.c_char_p
@@ -171,6 +176,16 @@ def dasgd_get_kernel_timing(ctx, which: int):
     return n.value, ms.value
 
 
+def dasgd_get_kernel_units(ctx, which: int) -> int:
+    n = ctypes.c_int64()
+    _check(_L.dasgd_get_kernel_units(ctx, which, ctypes.byref(n)), ctx)
+    return n.value
+
+
+def dasgd_refresh_lp(ctx):
+    _check(_L.dasgd_refresh_lp(ctx), ctx)
+
+
 def dasgd_reset_timing(ctx):
     _check(_L.dasgd_reset_timing(ctx), ctx)
 
@@ -240,7 +255,7 @@ class DaSGD:
 
     def __init__(self, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=DASGD_F32,
                  merge_mode=DASGD_MERGE_XI, flags=0, n_slots=None, ld=None, device=0, host_staging=False,
-                 sync_timeout_ms=0, order_after_current=True, snapshot_arrays=True):
+                 sync_timeout_ms=0, order_after_current=True, snapshot_arrays=True, n_chunks=0):
         if not torch.cuda.is_available():
             raise RuntimeError("DaSGD needs a CUDA device; there is no CPU implementation")
         self.K, self.P, self.tau, self.d = K, P, tau, d
@@ -279,8 +294,10 @@ class DaSGD:
         cfg.mean = self.mean.data_ptr()
         cfg.g_stage = self.g_stage.data_ptr() if self.g_stage is not None else None
         cfg.n_stage = n_stage
+        cfg.n_chunks = n_chunks
         cfg.main_stream, cfg.side_stream = self.main.cuda_stream, self.side.cuda_stream
         self.cfg = cfg
+        self._host_refs = []
         torch.cuda.synchronize(dev)  # the zero fills above ran on torch's current stream
         self.ctx = dasgd_init(cfg)
 
@@ -302,15 +319,20 @@ class DaSGD:
         self.w[:, :self.P] = w if w.dim() == 2 else w.unsqueeze(0)
         if m is not None and self.m is not None:
             self.m[:, :self.P] = torch.as_tensor(m, dtype=torch.float32, device=self.device)
-        if self.w_lp is not None:
-            self.w_lp.copy_(self.w)  # round-to-nearest-even cast
         torch.cuda.synchronize(self.device)
+        if self.w_lp is not None:
+            dasgd_refresh_lp(self.ctx)  # the library's own float32 -> bfloat16 rounding, on the main stream
+            self.sync()
 
     def _gptr(self, g: torch.Tensor) -> int:
         if self.order_after_current:
             self.main.wait_stream(torch.cuda.current_stream(self.device))
         if g.dtype != self.gdtype or tuple(g.shape) != (self.K, self.ld) or not g.is_contiguous() or not g.is_cuda:
             raise ValueError(f"gradients must be a contiguous CUDA {self.gdtype} tensor of shape {(self.K, self.ld)}")
+        # The kernels read g on the library's main stream, not on the stream torch allocated it on.  Telling
+        # the caching allocator keeps the block from being handed out again while they may still read it, so
+        # callers may pass temporaries (``eng.step(g_host.cuda(), lr)``).
+        g.record_stream(self.main)
         return g.data_ptr()
 
     # -- the path --------------------------------------------------------------
@@ -328,6 +350,7 @@ class DaSGD:
 
     def sync(self):
         dasgd_sync(self.ctx)
+        self._host_refs.clear()
 
     def step(self, g, lr):
         dasgd_step(self.ctx, self._gptr(g), lr)
@@ -336,6 +359,8 @@ class DaSGD:
         if g_host.is_cuda or g_host.dtype != self.gdtype or tuple(g_host.shape) != (self.K, self.ld):
             raise ValueError("step_host wants a host tensor shaped like the gradients")
         n = probe_host.numel() if probe_host is not None else 0
+        # the asynchronous copies read / write these host tensors until the next sync: keep them alive
+        self._host_refs.append((g_host, probe_host))
         dasgd_step_host(self.ctx, g_host.data_ptr(), lr, probe_host.data_ptr() if n else None, n)
 
     # -- introspection ---------------------------------------------------------
@@ -362,6 +387,10 @@ class DaSGD:
     def kernel_timing(self):
         """{kind: (launches, total ms)} for the five kinds of timed work."""
         return {name: dasgd_get_kernel_timing(self.ctx, i) for i, name in enumerate(self.KERNELS)}
+
+    def kernel_units(self):
+        """{kind: replica-parameters processed by the timed launches of that kind}."""
+        return {name: dasgd_get_kernel_units(self.ctx, i) for i, name in enumerate(self.KERNELS)}
 
     def reset_timing(self):
         dasgd_reset_timing(self.ctx)

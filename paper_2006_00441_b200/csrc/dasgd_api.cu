@@ -26,17 +26,28 @@ struct Slot {
   int64_t s = 0;                 // completed local steps when the snapshot was taken
   cudaEvent_t e_snap = nullptr;  // main stream: snapshot written
   cudaEvent_t e_avg = nullptr;   // side stream: mean written
+  int stall_sp = -1;             // timing: span whose ev[1] marks "mean complete" (-1: none)
+  std::vector<int> stall_sp_c;   // the same per column range
   int buf = -1;                  // index into ctx->pool of the array that holds this snapshot
   bool holds = false;            // this slot still keeps pool[buf] from being overwritten
+  // Chunked pipeline (n_chunks > 1): one event pair per column range.  `chunked` says which set the
+  // last snapshot of this slot recorded.
+  std::vector<cudaEvent_t> e_snap_c, e_avg_c;
+  bool chunked = false;
 };
 
-// A pair of timing events around one piece of stream work, tagged with what it measures.
+// A pair of timing events, tagged with what the time between them measures.  For the four kinds of
+// kernels the pair brackets the launch on its stream.  For TAG_STALL the pair straddles two streams:
+// ev[0] is recorded on the stream that is about to wait for a mean (it completes when that stream has
+// nothing else left to do), ev[1] on the side stream right after the mean kernel; ev[1] - ev[0], when
+// positive, is how long the mean kept that stream waiting.
 enum SpanTag { TAG_STEP = 0, TAG_SNAPSHOT = 1, TAG_MEAN = 2, TAG_MERGE = 3, TAG_STALL = 4, TAG_COUNT = 5 };
 struct Span {
   cudaEvent_t ev[2] = {nullptr, nullptr};
   int tag = 0;
-  bool open = false;   // begin recorded, not yet harvested
-  bool ended = false;  // end recorded
+  bool open = false;            // in use, not yet harvested
+  bool rec[2] = {false, false}; // which of the two events have been recorded
+  long long units = 0;          // replica-parameters the timed launch processes
 };
 
 struct DeviceGuard {
@@ -70,6 +81,15 @@ struct dasgd_ctx {
   std::vector<int> frozen;
   int cur = 0;
   bool rotate = false;
+  // Chunked pipeline: the parameter axis cut into `chunks` ranges of `chunk_cols` columns (a multiple
+  // of the vector kernels' tile, so every range starts on a 16-byte boundary); the last may be shorter.
+  int chunks = 1;
+  long long chunk_cols = 0;
+  // DASGD_FLAG_TWO_LANES: odd column ranges run on this stream, forked from and joined to the main
+  // stream inside every chunked iteration, so that the kernel of range i+1 fills the SMs as the kernel
+  // of range i drains instead of waiting for the stream's next command.
+  cudaStream_t s_lane = nullptr;
+  cudaEvent_t e_fork = nullptr, e_join = nullptr;
   // host-gradient staging (dasgd_step_host): a copy stream and, per staging array, an event for
   // "copy landed" (copy stream) and one for "kernels have consumed it" (main stream)
   cudaStream_t s_copy = nullptr;
@@ -79,6 +99,7 @@ struct dasgd_ctx {
   std::vector<Span> spans;
   int64_t span_n[TAG_COUNT] = {0, 0, 0, 0, 0};
   double span_ms[TAG_COUNT] = {0, 0, 0, 0, 0};
+  int64_t span_units[TAG_COUNT] = {0, 0, 0, 0, 0};
   std::string err;
 };
 
@@ -101,7 +122,11 @@ dasgd_status cuda_fail(dasgd_ctx *c, cudaError_t e, const char *what) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-float *snap_ptr(const dasgd_ctx *c, int slot) { return c->pool[c->slots[slot].buf]; }
+// The snapshot array of a slot; NULL for a slot that has none (made by the inline-mean schedule).
+float *snap_ptr(const dasgd_ctx *c, int slot) {
+  const int b = c->slots[slot].buf;
+  return b >= 0 && b < (int)c->pool.size() ? c->pool[b] : nullptr;
+}
 float *mean_ptr(const dasgd_ctx *c, int slot) {
   return static_cast<float *>(c->cfg.mean) + (size_t)slot * c->cfg.ld;
 }
@@ -126,28 +151,51 @@ Params base_params(const dasgd_ctx *c) {
 
 unsigned blocks_for(long long n, long long per_block) { return (unsigned)((n + per_block - 1) / per_block); }
 
+// The same operation restricted to the columns [col0, col0 + len) of every row: all pointers move by
+// col0 elements, the row stride stays.
+Params columns(const dasgd_ctx *c, Params p, long long col0, long long len) {
+  const size_t gsz = c->cfg.dtype == DASGD_BF16_MASTER_F32 ? 2 : 4;
+  p.w += col0;
+  p.w_out += col0;
+  if (p.m) p.m += col0;
+  if (p.g) p.g = static_cast<const char *>(p.g) + (size_t)col0 * gsz;
+  if (p.w_lp) p.w_lp += col0;
+  if (p.snap_out) p.snap_out += col0;
+  if (p.snap_in) p.snap_in += col0;
+  if (p.mean) p.mean += col0;
+  if (p.mean_out) p.mean_out += col0;
+  p.P = len;
+  return p;
+}
+
 // -------------------------------------------------------------- timing bookkeeping
 
 void harvest(dasgd_ctx *c, bool block) {
   for (Span &sp : c->spans) {
-    if (!sp.open || !sp.ended) continue;
-    if (block) {
-      if (cudaEventSynchronize(sp.ev[1]) != cudaSuccess) continue;
-    } else if (cudaEventQuery(sp.ev[1]) != cudaSuccess) {
-      cudaGetLastError();  // "not ready" is not an error here
-      continue;
+    if (!sp.open || !sp.rec[0] || !sp.rec[1]) continue;
+    bool ready = true;
+    for (int j = 0; j < 2 && ready; ++j) {
+      if (block) {
+        ready = cudaEventSynchronize(sp.ev[j]) == cudaSuccess;
+      } else if (cudaEventQuery(sp.ev[j]) != cudaSuccess) {
+        cudaGetLastError();  // "not ready" is not an error here
+        ready = false;
+      }
     }
+    if (!ready) continue;
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, sp.ev[0], sp.ev[1]) == cudaSuccess) {
+      if (sp.tag == TAG_STALL && ms < 0.f) ms = 0.f;  // the mean was complete before anyone waited
       c->span_n[sp.tag] += 1;
       c->span_ms[sp.tag] += ms;
+      c->span_units[sp.tag] += sp.units;
     }
-    sp.open = sp.ended = false;
+    sp.open = sp.rec[0] = sp.rec[1] = false;
   }
 }
 
-// Records the opening event of a span on `stream`; returns its index, or -1 when timing is off.
-int span_begin(dasgd_ctx *c, int tag, cudaStream_t stream) {
+// A free span (events created on demand); -1 when timing is off or events cannot be created.
+int span_alloc(dasgd_ctx *c, int tag, long long units) {
   if (!(c->cfg.flags & DASGD_FLAG_TIMING)) return -1;
   harvest(c, false);
   int idx = -1;
@@ -160,23 +208,53 @@ int span_begin(dasgd_ctx *c, int tag, cudaStream_t stream) {
     idx = (int)c->spans.size() - 1;
   }
   Span &sp = c->spans[idx];
-  if (cudaEventRecord(sp.ev[0], stream) != cudaSuccess) return -1;
   sp.tag = tag;
+  sp.units = units;
   sp.open = true;
-  sp.ended = false;
+  sp.rec[0] = sp.rec[1] = false;
   return idx;
 }
 
-void span_end(dasgd_ctx *c, int idx, cudaStream_t stream) {
+void span_record(dasgd_ctx *c, int idx, int which, cudaStream_t stream) {
   if (idx < 0) return;
-  if (cudaEventRecord(c->spans[idx].ev[1], stream) == cudaSuccess) c->spans[idx].ended = true;
-  else c->spans[idx].open = false;
+  Span &sp = c->spans[idx];
+  if (cudaEventRecord(sp.ev[which], stream) == cudaSuccess) sp.rec[which] = true;
+  else sp.open = false;
+}
+
+// Brackets a launch: records the opening event on `stream`; returns the span, or -1 when timing is off.
+int span_begin(dasgd_ctx *c, int tag, cudaStream_t stream, long long units = 0) {
+  const int idx = span_alloc(c, tag, units);
+  span_record(c, idx, 0, stream);
+  return idx;
+}
+
+void span_end(dasgd_ctx *c, int idx, cudaStream_t stream) { span_record(c, idx, 1, stream); }
+
+// Stall accounting.  mean_done: called right after a mean kernel has been put on the side stream; the
+// returned span is kept in the slot.  about_to_wait: called where `stream` is about to wait for that mean.
+int stall_mean_done(dasgd_ctx *c, int old_idx) {
+  if (old_idx >= 0 && old_idx < (int)c->spans.size() && c->spans[old_idx].open && c->spans[old_idx].tag == TAG_STALL &&
+      !c->spans[old_idx].rec[0])
+    c->spans[old_idx].open = false;  // the previous mean of this slot was never waited for
+  const int idx = span_alloc(c, TAG_STALL, 0);
+  span_record(c, idx, 1, c->s1);
+  return idx;
+}
+
+void stall_about_to_wait(dasgd_ctx *c, int &idx, cudaStream_t stream) {
+  if (idx >= 0 && idx < (int)c->spans.size() && c->spans[idx].open && c->spans[idx].tag == TAG_STALL && !c->spans[idx].rec[0])
+    span_record(c, idx, 0, stream);
+  idx = -1;
 }
 
 // -------------------------------------------------------------- kernel launchers
 
+// One launch enumerates (row, tile of 4096 columns) pairs in blockIdx.x.
+bool fits_one_launch(const Params &p) { return ((p.P + 4095) / 4096) * (long long)p.K <= 0x7FFFFFFFLL; }
+
 template <bool BF16, bool MOM, int MERGE, bool SNAP>
-dasgd_status launch_step_t(dasgd_ctx *c, const Params &p, bool vec) {
+dasgd_status launch_step_t(dasgd_ctx *c, const Params &p, bool vec, cudaStream_t stream) {
   constexpr int EPU = BF16 ? 8 : 4;
   constexpr int UNROLL = BF16 ? 2 : 4;
   long long done = 0;
@@ -184,15 +262,14 @@ dasgd_status launch_step_t(dasgd_ctx *c, const Params &p, bool vec) {
     const long long units = p.P / EPU;
     if (units > 0) {
       const long long tiles = (units + (long long)kThreads * UNROLL - 1) / ((long long)kThreads * UNROLL);
-      if (tiles * p.K > 0x7FFFFFFFLL) return fail(c, DASGD_ERR_UNSUPPORTED, "K*P too large for one launch");
-      dasgd::k_local_step_vec<BF16, MOM, MERGE, SNAP><<<(unsigned)(tiles * p.K), kThreads, 0, c->s0>>>(p);
+      dasgd::k_local_step_vec<BF16, MOM, MERGE, SNAP><<<(unsigned)(tiles * p.K), kThreads, 0, stream>>>(p);
       c->launches++;
     }
     done = units * EPU;
   }
   if (done < p.P) {
     dim3 grid(blocks_for(p.P - done, kThreads), (unsigned)p.K);
-    dasgd::k_local_step_scalar<BF16, MOM, MERGE, SNAP><<<grid, kThreads, 0, c->s0>>>(p, done);
+    dasgd::k_local_step_scalar<BF16, MOM, MERGE, SNAP><<<grid, kThreads, 0, stream>>>(p, done);
     c->launches++;
   }
   CU(c, cudaGetLastError());
@@ -200,37 +277,39 @@ dasgd_status launch_step_t(dasgd_ctx *c, const Params &p, bool vec) {
 }
 
 template <bool BF16, bool MOM>
-dasgd_status launch_step_m(dasgd_ctx *c, const Params &p, bool vec, int merge, bool snap) {
+dasgd_status launch_step_m(dasgd_ctx *c, const Params &p, bool vec, int merge, bool snap, cudaStream_t stream) {
   switch (merge * 2 + (snap ? 1 : 0)) {
-    case 0: return launch_step_t<BF16, MOM, 0, false>(c, p, vec);
-    case 1: return launch_step_t<BF16, MOM, 0, true>(c, p, vec);
-    case 2: return launch_step_t<BF16, MOM, 1, false>(c, p, vec);
-    case 3: return launch_step_t<BF16, MOM, 1, true>(c, p, vec);
-    case 4: return launch_step_t<BF16, MOM, 2, false>(c, p, vec);
-    default: return launch_step_t<BF16, MOM, 2, true>(c, p, vec);
+    case 0: return launch_step_t<BF16, MOM, 0, false>(c, p, vec, stream);
+    case 1: return launch_step_t<BF16, MOM, 0, true>(c, p, vec, stream);
+    case 2: return launch_step_t<BF16, MOM, 1, false>(c, p, vec, stream);
+    case 3: return launch_step_t<BF16, MOM, 1, true>(c, p, vec, stream);
+    case 4: return launch_step_t<BF16, MOM, 2, false>(c, p, vec, stream);
+    default: return launch_step_t<BF16, MOM, 2, true>(c, p, vec, stream);
   }
 }
 
 // merge: 0 none, 1 xi, 2 delta (fused into the step kernel); snap: also write p.snap_out
-dasgd_status launch_step(dasgd_ctx *c, const Params &p, bool vec, int merge, bool snap) {
+// `stream`: the main stream, or the second lane of a chunked iteration.
+dasgd_status launch_step(dasgd_ctx *c, const Params &p, bool vec, int merge, bool snap, cudaStream_t stream) {
   const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32;
   const bool mom = c->cfg.momentum != 0.0f;
-  const int sp = span_begin(c, TAG_STEP, c->s0);
+  if (!fits_one_launch(p)) return fail(c, DASGD_ERR_UNSUPPORTED, "K*P too large for one launch");
+  const int sp = span_begin(c, TAG_STEP, stream, (long long)p.K * p.P);
   dasgd_status st;
-  if (bf16) st = mom ? launch_step_m<true, true>(c, p, vec, merge, snap) : launch_step_m<true, false>(c, p, vec, merge, snap);
-  else st = mom ? launch_step_m<false, true>(c, p, vec, merge, snap) : launch_step_m<false, false>(c, p, vec, merge, snap);
-  span_end(c, sp, c->s0);
+  if (bf16) st = mom ? launch_step_m<true, true>(c, p, vec, merge, snap, stream) : launch_step_m<true, false>(c, p, vec, merge, snap, stream);
+  else st = mom ? launch_step_m<false, true>(c, p, vec, merge, snap, stream) : launch_step_m<false, false>(c, p, vec, merge, snap, stream);
+  span_end(c, sp, stream);
   return st;
 }
 
 dasgd_status launch_snapshot(dasgd_ctx *c, const Params &p) {
-  const int sp = span_begin(c, TAG_SNAPSHOT, c->s0);
+  if (!fits_one_launch(p)) return fail(c, DASGD_ERR_UNSUPPORTED, "K*P too large for one launch");
+  const int sp = span_begin(c, TAG_SNAPSHOT, c->s0, (long long)p.K * p.P);
   long long done = 0;
   if (c->vec) {
     const long long units = p.P / 4;
     if (units > 0) {
       const long long tiles = (units + (long long)kThreads * 4 - 1) / ((long long)kThreads * 4);
-      if (tiles * p.K > 0x7FFFFFFFLL) return fail(c, DASGD_ERR_UNSUPPORTED, "K*P too large for one launch");
       dasgd::k_snapshot_vec<<<(unsigned)(tiles * p.K), kThreads, 0, c->s0>>>(p);
       c->launches++;
     }
@@ -247,7 +326,7 @@ dasgd_status launch_snapshot(dasgd_ctx *c, const Params &p) {
 }
 
 dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
-  const int sp = span_begin(c, TAG_MEAN, c->s1);
+  const int sp = span_begin(c, TAG_MEAN, c->s1, (long long)p.K * p.P);
   long long done = 0;
   if (c->vec) {
     const long long units = p.P / 4;
@@ -272,7 +351,7 @@ dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
 template <bool BF16, int MODE, bool SNAP>
 dasgd_status launch_merge_t(dasgd_ctx *c, const Params &p) {
   constexpr int EPU = BF16 ? 8 : 4;
-  const int sp = span_begin(c, TAG_MERGE, c->s0);
+  const int sp = span_begin(c, TAG_MERGE, c->s0, (long long)p.K * p.P);
   long long done = 0;
   if (c->vec) {
     const long long units = p.P / EPU;
@@ -332,7 +411,7 @@ dasgd_status launch_allk_m(dasgd_ctx *c, const Params &p, bool vec, bool merge, 
 dasgd_status launch_allk(dasgd_ctx *c, const Params &p, bool vec, bool merge, bool meanout) {
   const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32;
   const bool mom = c->cfg.momentum != 0.0f;
-  const int sp = span_begin(c, TAG_STEP, c->s0);
+  const int sp = span_begin(c, TAG_STEP, c->s0, (long long)p.K * p.P);
   dasgd_status st;
   if (bf16) st = mom ? launch_allk_m<true, true>(c, p, vec, merge, meanout) : launch_allk_m<true, false>(c, p, vec, merge, meanout);
   else st = mom ? launch_allk_m<false, true>(c, p, vec, merge, meanout) : launch_allk_m<false, false>(c, p, vec, merge, meanout);
@@ -377,6 +456,7 @@ dasgd_status mark_snapped(dasgd_ctx *c, int slot, int buf) {
   Slot &sl = c->slots[slot];
   CU(c, cudaEventRecord(sl.e_snap, c->s0));
   sl.state = SLOT_SNAPPED;
+  sl.chunked = false;
   sl.s = c->t;
   sl.buf = buf;
   c->frozen[buf] += 1;
@@ -392,9 +472,15 @@ dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
   Slot &sl = c->slots[slot];
   if (sl.state != SLOT_AVERAGING)
     return fail(c, DASGD_ERR_BAD_STATE, "merge: the oldest snapshot has not been given to dasgd_average_async");
-  const int sp = span_begin(c, TAG_STALL, c->s0);
-  CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg, 0));
-  span_end(c, sp, c->s0);
+  if (sl.chunked) {
+    for (size_t i = 0; i < sl.e_avg_c.size(); ++i) {
+      stall_about_to_wait(c, sl.stall_sp_c[i], c->s0);
+      CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg_c[i], 0));
+    }
+  } else {
+    stall_about_to_wait(c, sl.stall_sp, c->s0);
+    CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg, 0));
+  }
   // From here on the main stream is ordered after the mean kernel.  The xi-blend no longer needs
   // the snapshot itself, so its array may be overwritten by what the main stream does next.
   if (c->cfg.merge_mode == DASGD_MERGE_XI && sl.holds) {
@@ -414,6 +500,16 @@ void release_oldest(dasgd_ctx *c) {
     sl.holds = false;
   }
   sl.state = SLOT_FREE;
+}
+
+void destroy_slot_events(Slot &sl) {
+  if (sl.e_snap) cudaEventDestroy(sl.e_snap);
+  if (sl.e_avg) cudaEventDestroy(sl.e_avg);
+  for (cudaEvent_t e : sl.e_snap_c) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : sl.e_avg_c) if (e) cudaEventDestroy(e);
+  sl.e_snap = sl.e_avg = nullptr;
+  sl.e_snap_c.clear();
+  sl.e_avg_c.clear();
 }
 
 bool merge_due(const dasgd_ctx *c, int64_t u) {
@@ -436,6 +532,7 @@ dasgd_status do_average(dasgd_ctx *c) {
   dasgd_status st = launch_reduce(c, p);
   if (st != DASGD_OK) return st;
   CU(c, cudaEventRecord(sl.e_avg, c->s1));
+  sl.stall_sp = stall_mean_done(c, sl.stall_sp);
   sl.state = SLOT_AVERAGING;
   return DASGD_OK;
 }
@@ -503,11 +600,32 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   if (c.n_stage < 0 || c.n_stage > 2) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: n_stage must be 0, 1 or 2");
   if ((c.n_stage > 0) != (c.g_stage != nullptr))
     return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: g_stage and n_stage must be given together");
+  if (c.n_chunks < 0 || c.n_chunks > 1024) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: n_chunks must be in [0, 1024]");
+  if (c.n_chunks > 1) {
+    const uint32_t need_flags = DASGD_FLAG_ROTATE_SNAPSHOT | DASGD_FLAG_FUSE_MERGE;
+    if ((c.flags & need_flags) != need_flags || inline_mean || c.d < 1)
+      return fail(nullptr, DASGD_ERR_INVALID_ARG,
+                  "init: n_chunks > 1 needs d >= 1, DASGD_FLAG_ROTATE_SNAPSHOT and DASGD_FLAG_FUSE_MERGE, and excludes "
+                  "DASGD_FLAG_INLINE_MEAN");
+  }
 
   int ndev = 0;
   cudaError_t e = cudaGetDeviceCount(&ndev);
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "init: cudaGetDeviceCount");
   if (c.device < 0 || c.device >= ndev) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: no such CUDA device");
+  for (const void *p : ptrs) {
+    if (!p) continue;
+    cudaPointerAttributes at{};
+    e = cudaPointerGetAttributes(&at, p);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return cuda_fail(nullptr, e, "init: cudaPointerGetAttributes");
+    }
+    if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged)
+      return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: w, m, w_lp, snap, mean and g_stage must be device memory");
+    if (at.type == cudaMemoryTypeDevice && at.device != c.device)
+      return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: a device buffer does not live on cfg.device");
+  }
 
   dasgd_ctx *ctx = new (std::nothrow) dasgd_ctx();
   if (!ctx) return fail(nullptr, DASGD_ERR_INVALID_ARG, "init: out of host memory");
@@ -521,18 +639,43 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   for (int i = 0; c.snap && i < c.n_slots; ++i)
     ctx->pool.push_back(static_cast<float *>(c.snap) + (size_t)i * c.K * c.ld);
   ctx->frozen.assign(ctx->pool.size(), 0);
+  if (c.n_chunks > 1 && c.d == 1) {  // only d == 1 needs the pipeline: for d >= 2 the mean has a whole step
+    const long long tile = 4096;     // columns per CTA of the vector step kernels, both dtypes
+    const long long tiles = (c.P + tile - 1) / tile;
+    const long long per = (tiles + c.n_chunks - 1) / c.n_chunks;
+    ctx->chunk_cols = per * tile;
+    ctx->chunks = (int)((c.P + ctx->chunk_cols - 1) / ctx->chunk_cols);
+  }
   DeviceGuard guard(c.device);
   ctx->slots.resize(c.n_slots);
   for (Slot &sl : ctx->slots) {
-    if ((e = cudaEventCreateWithFlags(&sl.e_snap, cudaEventDisableTiming)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&sl.e_avg, cudaEventDisableTiming)) != cudaSuccess) {
+    bool ok = (e = cudaEventCreateWithFlags(&sl.e_snap, cudaEventDisableTiming)) == cudaSuccess &&
+              (e = cudaEventCreateWithFlags(&sl.e_avg, cudaEventDisableTiming)) == cudaSuccess;
+    if (ok && ctx->chunks > 1) {
+      sl.e_snap_c.assign(ctx->chunks, nullptr);
+      sl.e_avg_c.assign(ctx->chunks, nullptr);
+      sl.stall_sp_c.assign(ctx->chunks, -1);
+      for (int i = 0; ok && i < ctx->chunks; ++i)
+        ok = (e = cudaEventCreateWithFlags(&sl.e_snap_c[i], cudaEventDisableTiming)) == cudaSuccess &&
+             (e = cudaEventCreateWithFlags(&sl.e_avg_c[i], cudaEventDisableTiming)) == cudaSuccess;
+    }
+    if (!ok) {
       dasgd_status st = cuda_fail(nullptr, e, "init: cudaEventCreate");
-      for (Slot &z : ctx->slots) {
-        if (z.e_snap) cudaEventDestroy(z.e_snap);
-        if (z.e_avg) cudaEventDestroy(z.e_avg);
-      }
+      for (Slot &z : ctx->slots) destroy_slot_events(z);
       delete ctx;
       return st;
+    }
+  }
+  if (ctx->chunks > 1 && (c.flags & DASGD_FLAG_TWO_LANES)) {
+    int prio = 0;
+    bool ok = cudaStreamGetPriority(ctx->s0, &prio) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&ctx->s_lane, cudaStreamNonBlocking, prio) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->e_fork, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->e_join, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      dasgd_destroy(ctx);
+      return fail(nullptr, DASGD_ERR_CUDA, "init: cannot create the second lane's stream and events");
     }
   }
   if (c.n_stage > 0) {
@@ -557,10 +700,7 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
   DeviceGuard guard(ctx->cfg.device);
   cudaStreamSynchronize(ctx->s0);
   cudaStreamSynchronize(ctx->s1);
-  for (Slot &sl : ctx->slots) {
-    if (sl.e_snap) cudaEventDestroy(sl.e_snap);
-    if (sl.e_avg) cudaEventDestroy(sl.e_avg);
-  }
+  for (Slot &sl : ctx->slots) destroy_slot_events(sl);
   for (Span &sp : ctx->spans)
     for (int j = 0; j < 2; ++j)
       if (sp.ev[j]) cudaEventDestroy(sp.ev[j]);
@@ -568,6 +708,12 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
     cudaStreamSynchronize(ctx->s_copy);
     cudaStreamDestroy(ctx->s_copy);
   }
+  if (ctx->s_lane) {
+    cudaStreamSynchronize(ctx->s_lane);
+    cudaStreamDestroy(ctx->s_lane);
+  }
+  if (ctx->e_fork) cudaEventDestroy(ctx->e_fork);
+  if (ctx->e_join) cudaEventDestroy(ctx->e_join);
   for (cudaEvent_t e : ctx->e_copied) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->e_consumed) if (e) cudaEventDestroy(e);
   delete ctx;
@@ -595,7 +741,7 @@ dasgd_status op_step(dasgd_ctx *c, const void *grads, float lr, int merge_slot, 
   p.w_out = c->pool[out];
   if (snap_buf >= 0) p.snap_out = c->pool[snap_buf];
   const int mode = merge_slot < 0 ? 0 : (c->cfg.merge_mode == DASGD_MERGE_DELTA ? 2 : 1);
-  dasgd_status st = launch_step(c, p, grads_vec_ok(c, grads), mode, snap_buf >= 0);
+  dasgd_status st = launch_step(c, p, grads_vec_ok(c, grads), mode, snap_buf >= 0, c->s0);
   if (st != DASGD_OK) return st;
   c->cur = out;
   c->t += 1;
@@ -650,6 +796,7 @@ dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, 
     if (c->slots[ms].state != SLOT_AVERAGING)
       return fail(c, DASGD_ERR_BAD_STATE, "step: the oldest snapshot has no mean yet");
     if (c->slots[ms].buf >= 0) {  // it came from dasgd_snapshot/dasgd_average_async: order after the side stream
+      stall_about_to_wait(c, c->slots[ms].stall_sp, c->s0);
       CU(c, cudaStreamWaitEvent(c->s0, c->slots[ms].e_avg, 0));
     }
     p.mean = mean_ptr(c, ms);
@@ -678,6 +825,104 @@ dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, 
       if (st != DASGD_OK) return st;
       release_oldest(c);
     }
+  }
+  return DASGD_OK;
+}
+
+// One iteration of the chunked pipeline (d == 1, rotating snapshots, merge folded into the step kernel).
+// Per column range i, on the main stream: wait for range i of the mean that lands (computed one
+// iteration ago, so normally long finished), run the step kernel on range i; if a snapshot is due,
+// record "range i written" and let the side stream average range i of the new weights while the main
+// stream goes on with ranges i+1, ...  The mean of range i thus has the rest of this iteration and the
+// first i ranges of the next one as its window (the condition t_c < d*t_p of Eq. 6, per range), although
+// the next iteration's kernels consume it directly.
+dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due, bool s_due) {
+  Params p = base_params(c);
+  p.g = grads;
+  p.lr = lr;
+  int ms = -1, ns = -1, reusable = -1;
+  bool per_chunk_wait = false;
+  if (m_due) {
+    if (c->pending.empty()) return fail(c, DASGD_ERR_BAD_STATE, "step: no snapshot is pending for the merge that is due");
+    ms = c->pending.front();
+    if (c->slots[ms].state != SLOT_AVERAGING)
+      return fail(c, DASGD_ERR_BAD_STATE, "step: the oldest snapshot has not been given to dasgd_average_async");
+  }
+  if (s_due) {
+    ns = find_free_slot(c);
+    if (ns < 0 && m_due) ns = ms;  // the slot whose mean this iteration consumes is refilled by it
+    if (ns < 0) return fail(c, DASGD_ERR_NO_SLOT, "step: every slot holds a pending average");
+  }
+  if (m_due) {
+    Slot &sl = c->slots[ms];
+    per_chunk_wait = sl.chunked;
+    if (!per_chunk_wait) {  // its mean came from dasgd_average_async: one event for the whole vector
+      stall_about_to_wait(c, sl.stall_sp, c->s0);
+      CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg, 0));
+    }
+    // Every kernel below that touches range i is ordered after the mean of range i, so the xi-blend no
+    // longer needs the snapshot array: it may be overwritten range by range.
+    if (c->cfg.merge_mode == DASGD_MERGE_XI && sl.holds) {
+      c->frozen[sl.buf] -= 1;
+      sl.holds = false;
+    }
+    p.mean = mean_ptr(c, ms);
+    p.snap_in = snap_ptr(c, ms);
+    reusable = reusable_buf(c, ms);
+  }
+  const int out = pick_w_out(c, reusable);
+  if (out < 0) return fail(c, DASGD_ERR_NO_SLOT, "step: no free weight array to write into");
+  p.w_out = c->pool[out];
+  Params q = base_params(c);  // the mean of the new snapshot = the array this iteration writes
+  if (s_due) {
+    q.snap_in = c->pool[out];
+    q.mean_out = mean_ptr(c, ns);
+  }
+  const int mode = !m_due ? 0 : (c->cfg.merge_mode == DASGD_MERGE_DELTA ? 2 : 1);
+  const bool vec = grads_vec_ok(c, grads);
+  // The mean of a range reads the weights its step kernel has just written: store them with the default
+  // cache policy so that part of them is still in L2 then (everything else streams through).
+  p.keep_w = s_due ? 1 : 0;
+  if (c->s_lane) {  // fork: the second lane starts after everything the main stream holds so far
+    CU(c, cudaEventRecord(c->e_fork, c->s0));
+    CU(c, cudaStreamWaitEvent(c->s_lane, c->e_fork, 0));
+  }
+  for (int i = 0; i < c->chunks; ++i) {
+    const long long col0 = (long long)i * c->chunk_cols;
+    const long long len = c->cfg.P - col0 < c->chunk_cols ? c->cfg.P - col0 : c->chunk_cols;
+    cudaStream_t lane = (c->s_lane && (i & 1)) ? c->s_lane : c->s0;
+    if (per_chunk_wait) {
+      stall_about_to_wait(c, c->slots[ms].stall_sp_c[i], lane);
+      CU(c, cudaStreamWaitEvent(lane, c->slots[ms].e_avg_c[i], 0));
+    }
+    dasgd_status st = launch_step(c, columns(c, p, col0, len), vec, mode, false, lane);
+    if (st != DASGD_OK) return st;
+    if (s_due) {
+      Slot &sl = c->slots[ns];
+      CU(c, cudaEventRecord(sl.e_snap_c[i], lane));
+      CU(c, cudaStreamWaitEvent(c->s1, sl.e_snap_c[i], 0));
+      st = launch_reduce(c, columns(c, q, col0, len));
+      if (st != DASGD_OK) return st;
+      CU(c, cudaEventRecord(sl.e_avg_c[i], c->s1));
+      sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
+    }
+  }
+  if (c->s_lane) {  // join: what the caller puts on the main stream next comes after both lanes
+    CU(c, cudaEventRecord(c->e_join, c->s_lane));
+    CU(c, cudaStreamWaitEvent(c->s0, c->e_join, 0));
+  }
+  c->cur = out;
+  c->t += 1;
+  if (m_due) release_oldest(c);
+  if (s_due) {
+    Slot &sl = c->slots[ns];
+    sl.state = SLOT_AVERAGING;
+    sl.chunked = true;
+    sl.s = c->t;
+    sl.buf = out;
+    c->frozen[out] += 1;
+    sl.holds = true;
+    c->pending.push_back(ns);
   }
   return DASGD_OK;
 }
@@ -724,7 +969,9 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
   const bool m_due = merge_due(ctx, u);
   const bool s_due = (u % cfg.tau) == 0;
   if (cfg.flags & DASGD_FLAG_INLINE_MEAN) return step_inline(ctx, grads, lr, m_due, s_due);
-  const bool fuse_merge = m_due && (cfg.flags & DASGD_FLAG_FUSE_MERGE) && cfg.d >= 2;
+  if (ctx->chunks > 1 && (m_due || s_due)) return step_chunked(ctx, grads, lr, m_due, s_due);
+  const bool fuse_merge = m_due && (cfg.flags & DASGD_FLAG_FUSE_MERGE) &&
+                          (cfg.d >= 2 || (cfg.d == 1 && (cfg.flags & DASGD_FLAG_FUSE_MERGE_D1)));
   // copy mode only: let the kernel that last writes w in this iteration also store the snapshot
   const bool fuse_snap = s_due && !ctx->rotate && (cfg.flags & DASGD_FLAG_FUSE_SNAPSHOT);
   dasgd_status st;
@@ -812,6 +1059,7 @@ dasgd_status dasgd_sync(dasgd_ctx *ctx) {
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(ctx->cfg.sync_timeout_ms);
   std::vector<cudaStream_t> streams = {ctx->s0, ctx->s1};
   if (ctx->s_copy) streams.push_back(ctx->s_copy);
+  if (ctx->s_lane) streams.push_back(ctx->s_lane);
   for (cudaStream_t s : streams) {
     for (;;) {
       cudaError_t e = cudaStreamQuery(s);
@@ -880,7 +1128,7 @@ dasgd_status dasgd_reset_timing(dasgd_ctx *ctx) {
   if (st != DASGD_OK) return st;
   DeviceGuard guard(ctx->cfg.device);
   harvest(ctx, true);
-  for (int i = 0; i < TAG_COUNT; ++i) { ctx->span_n[i] = 0; ctx->span_ms[i] = 0.0; }
+  for (int i = 0; i < TAG_COUNT; ++i) { ctx->span_n[i] = 0; ctx->span_ms[i] = 0.0; ctx->span_units[i] = 0; }
   return DASGD_OK;
 }
 
@@ -954,6 +1202,7 @@ dasgd_status dasgd_import_state(dasgd_ctx *ctx, const void *host_buf, int64_t le
     sl.state = (SlotState)q.state;   // the exporter had synchronised: a started mean is a finished mean,
     sl.s = q.s;                      // so its (never recorded) event makes the later wait a no-op
     sl.buf = q.buf;
+    sl.chunked = false;
     sl.holds = q.buf >= 0;
     if (sl.holds) ctx->frozen[q.buf] += 1;
     ctx->pending.push_back(q.slot);
@@ -992,6 +1241,41 @@ dasgd_status dasgd_advise_delay(dasgd_ctx *ctx, double extra_tp_ms, int32_t *d, 
   if (t_c_ms) *t_c_ms = tc;
   if (t_p_ms) *t_p_ms = tp;
   if (dasgd_delay_guideline(tc, tp, d, tau) != DASGD_OK) return fail(ctx, DASGD_ERR_INVALID_ARG, "advise_delay: degenerate timings");
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_kernel_units(dasgd_ctx *ctx, int32_t which, int64_t *units) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (which < 0 || which >= TAG_COUNT || !units)
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "get_kernel_units: which must be in [0, 4] and units non-NULL");
+  if (!(ctx->cfg.flags & DASGD_FLAG_TIMING))
+    return fail(ctx, DASGD_ERR_BAD_STATE, "get_kernel_units: DASGD_FLAG_TIMING not set");
+  dasgd_status st = dasgd_sync(ctx);
+  if (st != DASGD_OK) return st;
+  DeviceGuard guard(ctx->cfg.device);
+  harvest(ctx, true);
+  *units = ctx->span_units[which];
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_refresh_lp(dasgd_ctx *ctx) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (ctx->cfg.dtype != DASGD_BF16_MASTER_F32) return fail(ctx, DASGD_ERR_BAD_STATE, "refresh_lp: float32 mode has no w_lp");
+  DeviceGuard guard(ctx->cfg.device);
+  Params p = base_params(ctx);
+  long long done = 0;
+  if (ctx->vec && p.P / 8 > 0) {
+    dim3 grid(blocks_for(p.P / 8, kThreads), (unsigned)p.K);
+    dasgd::k_refresh_lp_vec<<<grid, kThreads, 0, ctx->s0>>>(p);
+    ctx->launches++;
+    done = p.P / 8 * 8;
+  }
+  if (done < p.P) {
+    dim3 grid(blocks_for(p.P - done, kThreads), (unsigned)p.K);
+    dasgd::k_refresh_lp_scalar<<<grid, kThreads, 0, ctx->s0>>>(p, done);
+    ctx->launches++;
+  }
+  CU(ctx, cudaGetLastError());
   return DASGD_OK;
 }
 

@@ -43,6 +43,8 @@ struct Params {
   float lr, mu, lambda, xi, omx;
   int nesterov;      // 1: step along g' + mu*m instead of m
   int decoupled_wd;  // 1: weight decay is applied to the weights directly, not added to the gradient
+  int keep_w;        // 1: the new weights are about to be re-read (by the mean of this column range): store
+                     //    them with the default cache policy instead of the streaming one
 };
 
 // ---------------------------------------------------------------- memory helpers
@@ -164,7 +166,8 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
         DASGD_F4_APPLY(w, blend_delta(w.x, a.x, s.x), blend_delta(w.y, a.y, s.y), blend_delta(w.z, a.z, s.z),
                        blend_delta(w.w, a.w, s.w))
       }
-      st_stream(reinterpret_cast<float4 *>(p.w_out + row + e) + f, w);
+      if (p.keep_w) reinterpret_cast<float4 *>(p.w_out + row + e)[f] = w;
+      else st_stream(reinterpret_cast<float4 *>(p.w_out + row + e) + f, w);
       if (MOM) st_stream(reinterpret_cast<float4 *>(p.m + row + e) + f, m);
       if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + row + e) + f, w);
       w4[j][f] = w;
@@ -404,7 +407,9 @@ __global__ void __launch_bounds__(kThreads) k_merge_scalar(const Params p, long 
 // The mean therefore needs no snapshot array and no second pass over HBM.  Same arithmetic and the
 // same summation tree as the separate kernels, so the results are bit-identical to theirs.
 // mean (read) and mean_out (written) may be the same array: a thread reads its elements of the old
-// mean before it writes the new ones.
+// mean before it writes the new ones, and no other thread touches them.  Because the array may be
+// written by this very kernel, the old mean is fetched with ordinary loads, not through the read-only
+// data path (which requires memory that stays unmodified for the whole kernel).
 
 template <bool BF16, bool MOM, bool MERGE, bool MEANOUT>
 __global__ void __launch_bounds__(kThreads) k_step_allk_vec(const Params p) {
@@ -417,7 +422,7 @@ __global__ void __launch_bounds__(kThreads) k_step_allk_vec(const Params p) {
   float4 a[F4], acc[F4][4];
 #pragma unroll
   for (int f = 0; f < F4; ++f) {
-    if (MERGE) a[f] = __ldg(reinterpret_cast<const float4 *>(p.mean + e) + f);
+    if (MERGE) a[f] = reinterpret_cast<const float4 *>(p.mean + e)[f];
 #pragma unroll
     for (int q = 0; q < 4; ++q) acc[f][q] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
@@ -514,6 +519,31 @@ __global__ void __launch_bounds__(kThreads) k_step_allk_scalar(const Params p, l
   }
   if (MEANOUT)
     p.mean_out[col] = __fdiv_rn(__fadd_rn(__fadd_rn(acc[0], acc[1]), __fadd_rn(acc[2], acc[3])), (float)p.K);
+}
+
+// ---------------------------------------------------------------- bf16 copy of the master weights
+// w_lp <- round-to-nearest-even(w), the same conversion every kernel that writes w applies.
+
+__global__ void __launch_bounds__(kThreads) k_refresh_lp_vec(const Params p) {
+  const long long u = (long long)blockIdx.x * kThreads + threadIdx.x;
+  const int k = blockIdx.y;
+  if (u >= p.P / 8) return;
+  const long long off = (long long)k * p.ld + u * 8;
+  const float4 a = reinterpret_cast<const float4 *>(p.w + off)[0];
+  const float4 b = reinterpret_cast<const float4 *>(p.w + off)[1];
+  uint4 o;
+  o.x = pack_bf16x2(a.x, a.y);
+  o.y = pack_bf16x2(a.z, a.w);
+  o.z = pack_bf16x2(b.x, b.y);
+  o.w = pack_bf16x2(b.z, b.w);
+  *reinterpret_cast<uint4 *>(p.w_lp + off) = o;
+}
+
+__global__ void __launch_bounds__(kThreads) k_refresh_lp_scalar(const Params p, long long p0) {
+  const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
+  if (col >= p.P) return;
+  const long long i = (long long)blockIdx.y * p.ld + col;
+  p.w_lp[i] = __float2bfloat16_rn(p.w[i]);
 }
 
 }  // namespace dasgd

@@ -35,10 +35,10 @@ def to_oracle_grad(g: torch.Tensor, P: int) -> np.ndarray:
 
 
 def make_pair(B, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=0, merge_mode=0, flags=0,
-              ld=None, n_slots=None, w0=None):
+              ld=None, n_slots=None, w0=None, n_chunks=0):
     """A libdasgd instance and an oracle with the same configuration and start point."""
     gpu = B.DaSGD(K, P, tau, d, xi, momentum, weight_decay, dtype=dtype, merge_mode=merge_mode, flags=flags,
-                  ld=ld, n_slots=n_slots)
+                  ld=ld, n_slots=n_slots, n_chunks=n_chunks)
     cpu = OracleDaSGD(K, P, tau, d, xi, momentum, weight_decay, dtype=dtype, merge_mode=merge_mode,
                       nesterov=bool(flags & 0x20), decoupled_wd=bool(flags & 0x40))
     if w0 is not None:

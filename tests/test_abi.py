@@ -46,6 +46,8 @@ def _cfg(**kw):
     (dict(dtype=1), "needs w_lp"), (dict(dtype=7), "unknown dtype"), (dict(merge_mode=3), "unknown merge_mode"),
     (dict(w=0x1004), "16-byte"), (dict(side_stream=None), "must differ"), (dict(n_stage=3, g_stage=0x4000), "n_stage"),
     (dict(n_stage=1), "given together"), (dict(g_stage=0x4000), "given together"),
+    (dict(n_chunks=2), "n_chunks > 1 needs"), (dict(n_chunks=1025, flags=0x8 | 0x4), "n_chunks must"),
+    (dict(n_chunks=4, flags=0x8 | 0x4, d=0), "n_chunks > 1 needs"), (dict(n_chunks=-1), "n_chunks must"),
 ])
 def test_init_rejects_bad_configuration_before_touching_cuda(bad, frag):
     with pytest.raises(B.DasgdError) as e:

@@ -15,6 +15,11 @@ pytestmark = pytest.mark.gpu
 
 FUSE_SNAP, FUSE_MERGE, ROTATE, INLINE = 0x2, 0x4, 0x8, 0x10
 NESTEROV, DECOUPLED = 0x20, 0x40
+FUSE_D1, LANES = 0x80, 0x100
+# schedules of dasgd_step: (flags, n_chunks).  The chunked pipeline only changes anything when d == 1.
+SCHEDS = [(0, 0), (FUSE_SNAP, 0), (FUSE_MERGE, 0), (FUSE_SNAP | FUSE_MERGE, 0), (ROTATE, 0), (ROTATE | FUSE_MERGE, 0),
+          (ROTATE | FUSE_MERGE, 3), (ROTATE | FUSE_MERGE, 2), (ROTATE | FUSE_MERGE | LANES, 3), (ROTATE | FUSE_MERGE | FUSE_D1, 0), (FUSE_MERGE | FUSE_D1, 0),
+          (INLINE, 0)]
 # f32 vector tile = 256 threads * 4 units * 4 elements = 4096 elements; bf16 tile = 256*2*8 = 4096
 SIZES = [1, 3, 4, 7, 8, 1000, 4096, 3 * 4096 + 1029]
 
@@ -124,15 +129,18 @@ SCHEDULES = [(1, 1), (2, 1), (4, 1), (1, 2), (2, 2), (4, 2), (2, 3), (3, 0), (1,
 
 
 @pytest.mark.parametrize("tau,d", SCHEDULES)
-@pytest.mark.parametrize("flags", [0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE, INLINE])
+@pytest.mark.parametrize("flags,n_chunks", SCHEDS)
 @pytest.mark.parametrize("K,dtype,mode", [(4, 0, 0), (3, 1, 0), (8, 0, 1)])
-def test_free_running_100_steps(B, tau, d, flags, K, dtype, mode):
+def test_free_running_100_steps(B, tau, d, flags, n_chunks, K, dtype, mode):
     if flags & INLINE and mode == 1:
         pytest.skip("the inline-mean schedule has no delta merge")
+    if n_chunks and d < 1:
+        pytest.skip("chunks need d >= 1")
     P, T = 2 * 4096 + 77, 100
     ld = (P + 7) // 8 * 8
     w0 = inputs.shared_start(2, P, 0.02).numpy()
-    gpu, cpu = make_pair(B, K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld, w0=w0)
+    gpu, cpu = make_pair(B, K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld, w0=w0,
+                         n_chunks=n_chunks)
     gd = torch.bfloat16 if dtype else torch.float32
     for t in range(T):
         g = grads(7, t, K, P, 0.0316, gd, ld)
@@ -153,23 +161,28 @@ def test_free_running_100_steps(B, tau, d, flags, K, dtype, mode):
 @pytest.mark.parametrize("tau,d", SCHEDULES)
 @pytest.mark.parametrize("dtype,mode", [(0, 0), (1, 0), (0, 1)])
 def test_fused_schedules_are_bit_identical_to_unfused(B, tau, d, dtype, mode):
-    K, P, T = 4, 4096 + 13, 25
+    K, P, T = 4, 2 * 4096 + 13, 25
     ld = (P + 7) // 8 * 8
     w0 = inputs.shared_start(4, P, 0.02)
     gd = torch.bfloat16 if dtype else torch.float32
-    outs = []
-    for flags in (0, FUSE_SNAP, FUSE_MERGE, FUSE_SNAP | FUSE_MERGE, ROTATE, ROTATE | FUSE_MERGE) + ((INLINE,) if mode == 0 else ()):
-        gpu = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld)
+    outs = {}
+    for flags, n_chunks in SCHEDS:
+        if (flags & INLINE and mode != 0) or (n_chunks and d < 1):
+            continue
+        gpu = B.DaSGD(K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode, flags=flags, ld=ld, n_chunks=n_chunks)
         gpu.set_state(w0)
         for t in range(T):
             gpu.step(grads(9, t, K, P, 0.0316, gd, ld), 0.1)
         gpu.sync()
-        outs.append((gpu.w[:, :P].clone(), gpu.m[:, :P].clone(), gpu.launches))   # payload columns only
-    for w, m, _ in outs[1:]:
-        assert torch.equal(w, outs[0][0]) and torch.equal(m, outs[0][1])
+        outs[(flags, n_chunks)] = (gpu.w[:, :P].clone(), gpu.m[:, :P].clone(), gpu.launches)   # payload columns only
+    w_ref, m_ref, n_ref = outs[(0, 0)]
+    for key, (w, m, _) in outs.items():
+        assert torch.equal(w, w_ref) and torch.equal(m, m_ref), key
     if d >= 1:
-        assert outs[1][2] < outs[0][2]  # the fused snapshot removes launches
-        assert outs[4][2] < outs[0][2]  # so does the rotating snapshot
+        assert outs[(FUSE_SNAP, 0)][2] < n_ref   # the fused snapshot removes launches
+        assert outs[(ROTATE, 0)][2] < n_ref      # so does the rotating snapshot
+    if d == 1:                                   # and folding the d = 1 merge into the step kernel removes the merge kernels
+        assert outs[(ROTATE | FUSE_MERGE | FUSE_D1, 0)][2] < outs[(ROTATE | FUSE_MERGE, 0)][2]
 
 
 def test_unaligned_rows_and_gradient_pointer_take_the_scalar_path(B):
@@ -212,6 +225,79 @@ def test_explicit_calls_equal_step(B, flags):
             b.snapshot(); b.average_async()
     a.sync(); b.sync()
     assert torch.equal(a.w, b.w) and torch.equal(a.m, b.m)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_chunked_pipeline_mixes_with_the_explicit_calls(B, mode):
+    """A context with n_chunks > 1: snapshots taken by dasgd_step (one event per column range) may be merged by
+    dasgd_merge, and snapshots taken by the explicit calls (one event) may be merged by dasgd_step."""
+    K, P, tau, d, T = 3, 3 * 4096 + 50, 2, 1, 12
+    ld = (P + 7) // 8 * 8
+    w0 = inputs.shared_start(60, P, 0.1).numpy()
+    gpu, cpu = make_pair(B, K, P, tau, d, 0.25, 0.9, 1e-3, merge_mode=mode, flags=ROTATE | FUSE_MERGE | LANES, ld=ld, w0=w0, n_chunks=3)
+    for t in range(T):
+        g = grads(61, t, K, P, 0.05, torch.float32, ld)
+        u = t + 1
+        if t % 4 < 2:      # the library's scheduler
+            gpu.step(g, 0.1)
+        else:              # the same iteration spelled out with the explicit calls
+            gpu.local_step(g, 0.1)
+            if u - d >= tau and (u - d) % tau == 0:
+                gpu.merge()
+            if u % tau == 0:
+                gpu.snapshot(); gpu.average_async()
+        cpu.step(to_oracle_grad(g, P), 0.1)
+        assert gpu.n_pending == cpu.n_pending
+    w, m = state_of(gpu)
+    assert_close(w, cpu.w, TOL_RUN, "w"); assert_close(m, cpu.m, TOL_RUN, "m")
+
+
+def test_chunks_need_rotation_fused_merge_and_a_delay(B):
+    for kw in (dict(flags=ROTATE), dict(flags=FUSE_MERGE), dict(flags=ROTATE | FUSE_MERGE, d=0), dict(flags=ROTATE | FUSE_MERGE, n_chunks=1025)):
+        args = dict(K=2, P=64, tau=2, d=1, xi=0.25, n_chunks=4)
+        args.update(kw)
+        with pytest.raises(B.DasgdError) as e:
+            B.DaSGD(**args)
+        assert e.value.status == B.DASGD_ERR_INVALID_ARG and "n_chunks" in str(e.value)
+
+
+def test_pending_slot_of_the_inline_schedule_reports_no_snapshot_array(B):
+    K, P = 2, 5000
+    a = B.DaSGD(K, P, 2, 1, 0.25, flags=INLINE, snapshot_arrays=False)
+    g = torch.zeros(K, P, device="cuda")
+    a.step(g, 0.1); a.step(g, 0.1); a.sync()
+    assert a.n_pending == 1
+    s, snap, mean = B.dasgd_get_pending(a.ctx, 0)
+    assert s == 2 and snap is None and mean == a.mean[0].data_ptr()
+
+
+def test_init_rejects_buffers_that_are_not_on_the_device(B):
+    e0 = B.DaSGD(2, 64, 2, 1, 0.25)
+    cfg = B.dasgd_config.from_buffer_copy(e0.cfg)
+    host = torch.zeros(2 * 64).pin_memory()
+    cfg.w = host.data_ptr()
+    with pytest.raises(B.DasgdError) as e:
+        B.dasgd_init(cfg)
+    assert e.value.status == B.DASGD_ERR_INVALID_ARG and "device memory" in str(e.value)
+
+
+def test_refresh_lp_is_the_oracles_rounding(B):
+    """With equal float32 masters the library's bfloat16 copy equals the oracle's bit for bit."""
+    K, P = 3, 4096 + 21
+    r = np.random.default_rng(5)
+    W = (r.standard_normal((K, P)) * np.exp(r.uniform(-8, 8, (K, P)))).astype(np.float32)
+    W[0, :4] = [1.00390625, 1.01171875, -1.00390625, 3.0e-39]    # ties to even, and a denormal
+    gpu, cpu = make_pair(B, K, P, 2, 1, 0.25, 0.9, 0.0, dtype=1, ld=(P + 7) // 8 * 8, w0=W)
+    np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), cpu.w_lp)
+    g = grads(70, 0, K, P, 0.1, torch.bfloat16, gpu.ld)
+    gpu.set_state(torch.from_numpy(cpu.w))
+    gpu.local_step(g, 0.1); cpu.local_step(to_oracle_grad(g, P), 0.1)
+    gpu.set_state(torch.from_numpy(cpu.w))          # teacher-force the masters, then compare the copies
+    np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), cpu.w_lp)
+    f32 = B.DaSGD(2, 64, 2, 1, 0.25)
+    with pytest.raises(B.DasgdError) as e:
+        B.dasgd_refresh_lp(f32.ctx)
+    assert e.value.status == B.DASGD_ERR_BAD_STATE
 
 
 def test_inline_mean_needs_no_snapshot_arrays_and_refuses_delta(B):
@@ -292,6 +378,28 @@ def test_timing_reports_hidden_fraction(B):
     assert all(v[1] > 0 for k, v in kt.items() if k != "stall")
     gpu.reset_timing()
     assert gpu.kernel_timing()["local_step"] == (0, 0.0)
+
+
+def test_stall_accounting_sees_a_mean_that_blocks_and_one_that_does_not(B):
+    """d = 1 with the merge folded into an unchunked step kernel and back-to-back steps: the kernel of step s+1
+    cannot start before the mean of step s is complete, and the main stream has nothing else to do meanwhile,
+    so practically all of the mean's time is stall.  The chunked pipeline gives each range's mean a window."""
+    K, P = 8, 1 << 21
+    g = torch.zeros(K, P, device="cuda")
+    fracs = {}
+    for name, flags, n_chunks in (("blocking", ROTATE | FUSE_MERGE | FUSE_D1, 0), ("pipelined", ROTATE | FUSE_MERGE, 8)):
+        gpu = B.DaSGD(K, P, 1, 1, 0.25, 0.9, flags=flags | B.DASGD_FLAG_TIMING, n_chunks=n_chunks, order_after_current=False)
+        for _ in range(5):
+            gpu.step(g, 0.1)
+        gpu.reset_timing()
+        for _ in range(30):
+            gpu.step(g, 0.1)
+        n, ms_avg, ms_stall = gpu.timing()
+        kt = gpu.kernel_timing()
+        assert n == 30 * max(1, n_chunks) and kt["stall"][0] == n and ms_avg > 0
+        fracs[name] = ms_stall / ms_avg
+    assert fracs["blocking"] > 0.5
+    assert fracs["pipelined"] < fracs["blocking"]
 
 
 def test_sync_gives_up_after_its_timeout_and_the_context_survives(B):
