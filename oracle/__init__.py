@@ -59,6 +59,9 @@ def bind(path: str) -> ctypes.CDLL:
     L.oracle_dasgd_merge.argtypes = [vp]
     L.oracle_dasgd_step.argtypes = [vp, vp, f32]
     L.oracle_dasgd_set_variant.argtypes = [vp, i32, i32]
+    L.oracle_dasgd_set_shard.argtypes = [vp, i32]
+    L.oracle_dasgd_partial_sum.argtypes = [vp, vp]
+    L.oracle_dasgd_set_mean_from_sum.argtypes = [vp, vp]
     L.oracle_dasgd_threads.argtypes = []
     f64, pi32 = ctypes.c_double, ctypes.POINTER(i32)
     L.oracle_dasgd_delay_guideline.argtypes = [f64, f64, pi32, pi32]
@@ -189,3 +192,32 @@ class OracleDaSGD:
 
     def step(self, g, lr):
         self._chk(self._L.oracle_dasgd_step(self._h, _ptr(self._grad(g)), lr), "step")
+
+    # -- a shard of the worker axis -----------------------------------------
+    def set_shard(self, K_total):
+        """This object holds K of K_total workers; the mean then needs the partial sums of all shards."""
+        self._chk(self._L.oracle_dasgd_set_shard(self._h, K_total), "set_shard")
+        self.K_total = K_total
+
+    def partial_sum(self):
+        """float64 [P]: sum over this shard's workers of the oldest snapshot without a mean."""
+        out = np.empty((self.P,), np.float64)
+        self._chk(self._L.oracle_dasgd_partial_sum(self._h, _ptr(out)), "partial_sum")
+        return out
+
+    def set_mean_from_sum(self, total):
+        total = np.ascontiguousarray(total, dtype=np.float64)
+        assert total.shape == (self.P,)
+        self._chk(self._L.oracle_dasgd_set_mean_from_sum(self._h, _ptr(total)), "set_mean_from_sum")
+
+    def sharded_step(self, g, lr, exchange):
+        """One iteration of the schedule on a shard: `exchange(partial_sum) -> total` is the all-reduce."""
+        self.local_step(g, lr)
+        u = self.t
+        if self.d > 0 and u - self.d >= self.tau and (u - self.d) % self.tau == 0:
+            self.merge()
+        if u % self.tau == 0:
+            self.snapshot()
+            self.set_mean_from_sum(exchange(self.partial_sum()))
+            if self.d == 0:
+                self.merge()

@@ -43,6 +43,7 @@ struct Pending {
 
 struct oracle_dasgd {
   int32_t K, tau, d, dtype, merge_mode;
+  int32_t K_total = 0;  // > 0: this object holds K of the K_total workers (a shard of the worker axis)
   int64_t P;
   float xi, momentum, weight_decay;
   bool nesterov = false, decoupled_wd = false;
@@ -164,6 +165,7 @@ int oracle_dasgd_snapshot(oracle_dasgd *o) {
 // (1/M) * sum over workers, Eq. 2 second branch.
 int oracle_dasgd_average(oracle_dasgd *o) {
   if (!o) return ORACLE_ERR_ARG;
+  if (o->K_total > 0) return ORACLE_ERR_STATE;  // a shard cannot form the mean alone
   Pending *q = nullptr;
   for (auto &cand : o->pending)
     if (!cand.averaged) { q = &cand; break; }  // oldest snapshot that has no mean yet
@@ -176,6 +178,47 @@ int oracle_dasgd_average(oracle_dasgd *o) {
     for (int32_t k = 0; k < o->K; ++k) acc += static_cast<double>(q->snap[static_cast<size_t>(k) * P + p]);
     q->mean[p] = static_cast<float>(acc / static_cast<double>(o->K));
   }
+  q->averaged = true;
+  return ORACLE_OK;
+}
+
+// The worker axis split over several holders (the data-parallel deployment of Section II-B: every
+// machine owns some of the M workers and an all-reduce forms the sum).  The (1/M) * sum_j of Eq. 2 is
+// then a two-level sum: each holder adds up its own workers, the partial sums are added across
+// holders (by the caller), and the total is divided by M = K_total once.
+int oracle_dasgd_set_shard(oracle_dasgd *o, int32_t K_total) {
+  if (!o || K_total < o->K) return ORACLE_ERR_ARG;
+  o->K_total = K_total;
+  return ORACLE_OK;
+}
+
+int oracle_dasgd_partial_sum(const oracle_dasgd *o, double *sum) {
+  if (!o || !sum) return ORACLE_ERR_ARG;
+  const Pending *q = nullptr;
+  for (const auto &cand : o->pending)
+    if (!cand.averaged) { q = &cand; break; }  // oldest snapshot that has no mean yet
+  if (!q) return ORACLE_ERR_STATE;
+  const int64_t P = o->P;
+#pragma omp parallel for schedule(static)
+  for (int64_t p = 0; p < P; ++p) {
+    double acc = 0.0;
+    for (int32_t k = 0; k < o->K; ++k) acc += static_cast<double>(q->snap[static_cast<size_t>(k) * P + p]);
+    sum[p] = acc;
+  }
+  return ORACLE_OK;
+}
+
+int oracle_dasgd_set_mean_from_sum(oracle_dasgd *o, const double *total) {
+  if (!o || !total) return ORACLE_ERR_ARG;
+  if (o->K_total < 1) return ORACLE_ERR_STATE;
+  Pending *q = nullptr;
+  for (auto &cand : o->pending)
+    if (!cand.averaged) { q = &cand; break; }
+  if (!q) return ORACLE_ERR_STATE;
+  const int64_t P = o->P;
+  q->mean.assign(static_cast<size_t>(P), 0.0f);
+#pragma omp parallel for schedule(static)
+  for (int64_t p = 0; p < P; ++p) q->mean[p] = static_cast<float>(total[p] / static_cast<double>(o->K_total));
   q->averaged = true;
   return ORACLE_OK;
 }

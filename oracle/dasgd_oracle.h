@@ -77,6 +77,21 @@ int oracle_dasgd_snapshot(oracle_dasgd *o);
 int oracle_dasgd_average(oracle_dasgd *o); /* mean of the oldest snapshot not yet averaged */
 int oracle_dasgd_merge(oracle_dasgd *o);   /* blend the OLDEST pending mean, then drop it   */
 
+/* Sharded worker axis (the data-parallel setting of Section II-B, where the workers live on several
+ * machines and an all-reduce adds their contributions).  After oracle_dasgd_set_shard(o, K_total) the
+ * object holds K of the K_total workers of Eq. 2; oracle_dasgd_average and oracle_dasgd_step then
+ * fail with ORACLE_ERR_STATE, because the mean needs the other shards.  Instead:
+ *   oracle_dasgd_partial_sum      -- sum over this shard's workers of the oldest snapshot that has no
+ *                                    mean yet, per parameter, in double ([P]);
+ *   (the caller adds the partial sums of all shards)
+ *   oracle_dasgd_set_mean_from_sum -- mean = total / K_total, rounded to float32 once; the snapshot
+ *                                    then counts as averaged and oracle_dasgd_merge can blend it.
+ * Pinned: the shards of a partitioned run reproduce the unsharded oracle (a two-level sum of the same
+ * terms), one shard with K_total = K reproduces it bit for bit, and identical shards behave like one. */
+int oracle_dasgd_set_shard(oracle_dasgd *o, int32_t K_total);
+int oracle_dasgd_partial_sum(const oracle_dasgd *o, double *sum);
+int oracle_dasgd_set_mean_from_sum(oracle_dasgd *o, const double *total);
+
 /* One iteration of the schedule: local step; merge if one lands; snapshot+mean if due. */
 int oracle_dasgd_step(oracle_dasgd *o, const void *g, float lr);
 

@@ -10,6 +10,7 @@ import oracle
 from tests import test_oracle_golden as G
 from tests import test_delay_guideline as D
 from tests import test_oracle_invariants as I
+from tests import test_oracle_sharded as S
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "dasgd_oracle.cpp")
 
@@ -41,6 +42,11 @@ MUTATIONS = {
     "guideline: tau equals d": ("*tau = k + 1;", "*tau = k;"),
     "guideline: non-strict inequality": ("while (!(t_c < static_cast<double>(k) * t_p)) ++k;",
                                          "while (!(t_c <= static_cast<double>(k) * t_p)) ++k;"),
+    "sharded mean divided by the shard's own size": ("total[p] / static_cast<double>(o->K_total)", "total[p] / static_cast<double>(o->K)"),
+    "partial sum already divided": ("    sum[p] = acc;", "    sum[p] = acc / static_cast<double>(o->K);"),
+    "partial sum takes the newest snapshot": (
+        "  const Pending *q = nullptr;\n  for (const auto &cand : o->pending)\n    if (!cand.averaged) { q = &cand; break; }",
+        "  const Pending *q = nullptr;\n  for (const auto &cand : o->pending)\n    if (!cand.averaged) { q = &cand; }"),
     "momentum merged too": ("o->pending.pop_front();\n  return ORACLE_OK;", "for (auto &x : o->m) x *= o->xi;\n  o->pending.pop_front();\n  return ORACLE_OK;"),
 }
 
@@ -68,6 +74,10 @@ def battery():
     I.test_decoupled_weight_decay_closed_form_with_momentum()
     I.test_bf16_rounding_matches_torch_cast()
     I.test_bf16_mode_master_equals_f32_run_on_widened_gradients()
+    S.test_mean_divides_by_the_total_number_of_workers()
+    S.test_shards_in_one_process_reproduce_the_unsharded_oracle(2, 1, (3, 5))
+    S.test_one_shard_holding_every_worker_is_the_unsharded_oracle_bit_for_bit()
+    S.test_explicit_calls_on_shards_with_two_snapshots_in_flight()
     for row in D.table2():
         D.test_oracle_reproduces_table2(row)
     assert oracle.delay_guideline(1.0, 1.0) == (2, 3)      # Eq. 3 is strict: d > t_c / t_p
