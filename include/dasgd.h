@@ -247,6 +247,30 @@ dasgd_status dasgd_get_kernel_units(dasgd_ctx *ctx, int32_t which, int64_t *unit
  * no rounding of the method's state happens outside the library.  DASGD_ERR_BAD_STATE in float32 mode. */
 dasgd_status dasgd_refresh_lp(dasgd_ctx *ctx);
 
+/* ---- Sharded worker axis (the data-parallel setting of Section II-B: the M workers live on several GPUs
+ * and an all-reduce adds their contributions; Section III: the averaging runs while the local steps go on).
+ *
+ * A context then holds cfg.K of K_total workers.  Where the other entry points form the mean, such a
+ * context (1) writes the plain float32 SUM of its own rows into the mean slot (skipped when cfg.K == 1: the
+ * row is its own sum), (2) calls `exchange`, which must leave in recv_device the element-wise sum of
+ * send_device over ALL shards, ordered on side_stream (an all-reduce enqueued on that stream), and
+ * (3) divides by K_total, correctly rounded, where the merge reads the result.  The mean slots (and
+ * dasgd_get_pending) therefore hold sums, not means.  Every shard must issue the same sequence of calls.
+ * Call dasgd_set_shard right after dasgd_init.  Not available with DASGD_FLAG_INLINE_MEAN. */
+typedef dasgd_status (*dasgd_exchange_fn)(void *user, const void *send_device, void *recv_device, int64_t count,
+                                          void *side_stream);
+dasgd_status dasgd_set_shard(dasgd_ctx *ctx, int32_t K_total, dasgd_exchange_fn exchange, void *user);
+
+/* The exchange over NCCL: ncclAllReduce(sum, float32) on the side stream.  The NCCL library (libnccl.so.2) is
+ * loaded on first use; DASGD_ERR_UNSUPPORTED if it cannot be.  Rank 0 makes an id (128 bytes, host) and hands
+ * it to the other ranks by any means; every rank then creates its communicator with the device current that
+ * owns its context, and passes it to dasgd_set_shard_nccl.  The communicator stays the caller's: destroy it
+ * after the context. */
+dasgd_status dasgd_nccl_unique_id(void *id128_host);
+dasgd_status dasgd_nccl_comm_init(void **comm, const void *id128_host, int32_t nranks, int32_t rank, int32_t device);
+dasgd_status dasgd_nccl_comm_destroy(void *comm);
+dasgd_status dasgd_set_shard_nccl(dasgd_ctx *ctx, int32_t K_total, void *comm);
+
 /* Number of kernels this context has launched so far. */
 dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches);
 

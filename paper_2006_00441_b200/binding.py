@@ -35,7 +35,11 @@ EXPORTS = [
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
     "dasgd_average_merge_noalloc", "dasgd_delay_guideline", "dasgd_advise_delay", "dasgd_export_state", "dasgd_import_state",
     "dasgd_get_kernel_units", "dasgd_refresh_lp",
+    "dasgd_set_shard", "dasgd_set_shard_nccl", "dasgd_nccl_unique_id", "dasgd_nccl_comm_init", "dasgd_nccl_comm_destroy",
 ]
+
+# dasgd_exchange_fn: (user, send_device, recv_device, count, side_stream) -> status
+EXCHANGE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p)
 
 
 class dasgd_config(ctypes.Structure):
@@ -92,6 +96,11 @@ def _load() -> ctypes.CDLL:
     L.dasgd_advise_delay.argtypes = [vp, f64, pi32, pi32, pf64, pf64]
     L.dasgd_export_state.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
     L.dasgd_import_state.argtypes = [vp, vp, i64]
+    L.dasgd_set_shard.argtypes = [vp, i32, EXCHANGE_FN, vp]
+    L.dasgd_set_shard_nccl.argtypes = [vp, i32, vp]
+    L.dasgd_nccl_unique_id.argtypes = [vp]
+    L.dasgd_nccl_comm_init.argtypes = [ctypes.POINTER(vp), vp, i32, i32, i32]
+    L.dasgd_nccl_comm_destroy.argtypes = [vp]
     L.dasgd_version.argtypes = []
     L.dasgd_version.restype = ctypes.c_char_p
     return L
@@ -215,6 +224,31 @@ def dasgd_export_state(ctx) -> bytes:
 
 def dasgd_import_state(ctx, blob: bytes):
     _check(_L.dasgd_import_state(ctx, blob, len(blob)), ctx)
+
+
+def dasgd_set_shard(ctx, K_total: int, exchange, user=None):
+    """`exchange`: an EXCHANGE_FN instance; the caller keeps it alive as long as the context."""
+    _check(_L.dasgd_set_shard(ctx, K_total, exchange, user), ctx)
+
+
+def dasgd_set_shard_nccl(ctx, K_total: int, comm):
+    _check(_L.dasgd_set_shard_nccl(ctx, K_total, comm), ctx)
+
+
+def dasgd_nccl_unique_id() -> bytes:
+    buf = ctypes.create_string_buffer(128)
+    _check(_L.dasgd_nccl_unique_id(buf), None)
+    return buf.raw
+
+
+def dasgd_nccl_comm_init(unique_id: bytes, nranks: int, rank: int, device: int) -> ctypes.c_void_p:
+    comm = ctypes.c_void_p()
+    _check(_L.dasgd_nccl_comm_init(ctypes.byref(comm), unique_id, nranks, rank, device), None)
+    return comm
+
+
+def dasgd_nccl_comm_destroy(comm):
+    _check(_L.dasgd_nccl_comm_destroy(comm), None)
 
 
 def dasgd_get_launches(ctx) -> int:
@@ -421,6 +455,24 @@ class DaSGD:
     @property
     def launches(self):
         return dasgd_get_launches(self.ctx)
+
+    # -- sharded worker axis ---------------------------------------------------
+    def set_shard(self, K_total, exchange=None, nccl_comm=None):
+        """This object holds K of K_total workers.  Either `nccl_comm` (from dasgd_nccl_comm_init) or
+        `exchange(send_ptr, recv_ptr, count, stream_ptr)`, a Python callable that enqueues the all-reduce of
+        the partial sums on the side stream."""
+        if nccl_comm is not None:
+            dasgd_set_shard_nccl(self.ctx, K_total, nccl_comm)
+        else:
+            def thunk(user, send, recv, count, stream):
+                try:
+                    exchange(send, recv, count, stream)
+                    return DASGD_OK
+                except Exception:
+                    return DASGD_ERR_CUDA
+            self._exchange = EXCHANGE_FN(thunk)      # keep the callback object alive
+            dasgd_set_shard(self.ctx, K_total, self._exchange, None)
+        self.K_total = K_total
 
     def close(self):
         if getattr(self, "ctx", None):

@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdasgd.so")
-SOURCES = [os.path.join(CSRC, "dasgd_api.cu"), os.path.join(CSRC, "dasgd_noalloc.cu")]
+SOURCES = [os.path.join(CSRC, "dasgd_api.cu"), os.path.join(CSRC, "dasgd_noalloc.cu"), os.path.join(CSRC, "dasgd_nccl.cu")]
 HEADERS = [os.path.join(CSRC, "dasgd_kernels.cuh"), os.path.join(ROOT, "include", "dasgd.h")]
 
 
@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += SOURCES + ["-o", LIB + ".tmp"]
+    cmd += SOURCES + ["-ldl", "-o", LIB + ".tmp"]
     subprocess.run(cmd, check=True)
     os.replace(LIB + ".tmp", LIB)
     return LIB

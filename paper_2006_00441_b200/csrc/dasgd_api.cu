@@ -90,6 +90,11 @@ struct dasgd_ctx {
   // of range i drains instead of waiting for the stream's next command.
   cudaStream_t s_lane = nullptr;
   cudaEvent_t e_fork = nullptr, e_join = nullptr;
+  // Sharded worker axis: this context holds cfg.K of K_total workers; `exchange` adds the partial sums of
+  // all shards (an all-reduce) on the side stream.  0 / NULL: every worker is here.
+  int32_t K_total = 0;
+  dasgd_exchange_fn exchange = nullptr;
+  void *exchange_user = nullptr;
   // host-gradient staging (dasgd_step_host): a copy stream and, per staging array, an event for
   // "copy landed" (copy stream) and one for "kernels have consumed it" (main stream)
   cudaStream_t s_copy = nullptr;
@@ -146,6 +151,7 @@ Params base_params(const dasgd_ctx *c) {
   p.decoupled_wd = (c->cfg.flags & DASGD_FLAG_DECOUPLED_WD) ? 1 : 0;
   p.xi = c->cfg.xi;
   p.omx = 1.0f - c->cfg.xi;
+  p.mean_div = c->K_total > 0 ? (float)c->K_total : 0.0f;
   return p;
 }
 
@@ -326,7 +332,6 @@ dasgd_status launch_snapshot(dasgd_ctx *c, const Params &p) {
 }
 
 dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
-  const int sp = span_begin(c, TAG_MEAN, c->s1, (long long)p.K * p.P);
   long long done = 0;
   if (c->vec) {
     const long long units = p.P / 4;
@@ -343,9 +348,34 @@ dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
     dasgd::k_reduce_scalar<<<blocks_for(p.P - done, kThreads), kThreads, 0, c->s1>>>(p, done);
     c->launches++;
   }
-  span_end(c, sp, c->s1);
   CU(c, cudaGetLastError());
   return DASGD_OK;
+}
+
+// The worker-axis mean of the snapshot p.snap_in into p.mean_out, on the side stream.  With every worker
+// in this context: one kernel.  With a sharded worker axis: the kernel writes the plain sum of this
+// context's rows (no kernel when there is a single row: the row is its own sum), then the exchange adds
+// the sums of all shards in place; the division by the total number of workers happens where the merge
+// reads the result.
+dasgd_status launch_mean(dasgd_ctx *c, Params p) {
+  const int sp = span_begin(c, TAG_MEAN, c->s1, (long long)p.K * p.P);
+  dasgd_status st = DASGD_OK;
+  if (c->K_total == 0) {
+    st = launch_reduce(c, p);
+  } else {
+    const float *send = p.snap_in;
+    if (p.K > 1) {
+      p.sum_only = 1;
+      st = launch_reduce(c, p);
+      send = p.mean_out;
+    }
+    if (st == DASGD_OK) {
+      st = c->exchange(c->exchange_user, send, p.mean_out, p.P, c->s1);
+      if (st != DASGD_OK) fail(c, st, "average: the exchange of the partial sums failed");
+    }
+  }
+  span_end(c, sp, c->s1);
+  return st;
 }
 
 template <bool BF16, int MODE, bool SNAP>
@@ -529,7 +559,7 @@ dasgd_status do_average(dasgd_ctx *c) {
   Params p = base_params(c);
   p.snap_in = snap_ptr(c, slot);
   p.mean_out = mean_ptr(c, slot);
-  dasgd_status st = launch_reduce(c, p);
+  dasgd_status st = launch_mean(c, p);
   if (st != DASGD_OK) return st;
   CU(c, cudaEventRecord(sl.e_avg, c->s1));
   sl.stall_sp = stall_mean_done(c, sl.stall_sp);
@@ -901,7 +931,7 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
       Slot &sl = c->slots[ns];
       CU(c, cudaEventRecord(sl.e_snap_c[i], lane));
       CU(c, cudaStreamWaitEvent(c->s1, sl.e_snap_c[i], 0));
-      st = launch_reduce(c, columns(c, q, col0, len));
+      st = launch_mean(c, columns(c, q, col0, len));
       if (st != DASGD_OK) return st;
       CU(c, cudaEventRecord(sl.e_avg_c[i], c->s1));
       sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
@@ -1277,6 +1307,25 @@ dasgd_status dasgd_refresh_lp(dasgd_ctx *ctx) {
   }
   CU(ctx, cudaGetLastError());
   return DASGD_OK;
+}
+
+dasgd_status dasgd_set_shard(dasgd_ctx *ctx, int32_t K_total, dasgd_exchange_fn exchange, void *user) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (K_total < ctx->cfg.K || !exchange)
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "set_shard: need K_total >= K and an exchange function");
+  if (ctx->cfg.flags & DASGD_FLAG_INLINE_MEAN)
+    return fail(ctx, DASGD_ERR_UNSUPPORTED, "set_shard: the inline-mean schedule keeps every worker in one context");
+  if (ctx->t != 0 || !ctx->pending.empty())
+    return fail(ctx, DASGD_ERR_BAD_STATE, "set_shard: the context has already been used");
+  ctx->K_total = K_total;
+  ctx->exchange = exchange;
+  ctx->exchange_user = user;
+  return DASGD_OK;
+}
+
+// for the other translation units of the library (not exported)
+__attribute__((visibility("hidden"))) dasgd_status dasgd_internal_fail(dasgd_ctx *ctx, dasgd_status st, const char *msg) {
+  return fail(ctx, st, msg);
 }
 
 dasgd_status dasgd_get_launches(const dasgd_ctx *ctx, int64_t *launches) {

@@ -43,6 +43,9 @@ struct Params {
   float lr, mu, lambda, xi, omx;
   int nesterov;      // 1: step along g' + mu*m instead of m
   int decoupled_wd;  // 1: weight decay is applied to the weights directly, not added to the gradient
+  float mean_div;    // 0: `mean` holds the mean.  Otherwise `mean` holds the SUM over all workers (sharded
+                     //    worker axis) and the mean is that sum divided, correctly rounded, by this number
+  int sum_only;      // 1: the worker-axis kernel writes the plain sum of its K rows, not their mean
   int keep_w;        // 1: the new weights are about to be re-read (by the mean of this column range): store
                      //    them with the default cache policy instead of the streaming one
 };
@@ -76,6 +79,23 @@ __device__ __forceinline__ void step_elem(float &w, float &m, float g, const Par
   const float w_old = w;
   w = fmaf(-p.lr, dir, w);
   if (p.decoupled_wd) w = fmaf(-__fmul_rn(p.lr, p.lambda), w_old, w);
+}
+
+// The mean as the merge sees it: stored as such, or formed here from the all-worker sum.
+__device__ __forceinline__ float mean_of(float v, const Params &p) {
+  return p.mean_div != 0.0f ? __fdiv_rn(v, p.mean_div) : v;
+}
+__device__ __forceinline__ float4 mean_of(float4 v, const Params &p) {
+  if (p.mean_div != 0.0f) {
+    v.x = __fdiv_rn(v.x, p.mean_div); v.y = __fdiv_rn(v.y, p.mean_div);
+    v.z = __fdiv_rn(v.z, p.mean_div); v.w = __fdiv_rn(v.w, p.mean_div);
+  }
+  return v;
+}
+
+// Sum of the K rows -> what the worker-axis kernel stores.
+__device__ __forceinline__ float finish_mean(float s, float kf, const Params &p) {
+  return p.sum_only ? s : __fdiv_rn(s, kf);
 }
 
 __device__ __forceinline__ float blend_xi(float w, float mean, const Params &p) {
@@ -139,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
       for (int f = 0; f < F4; ++f) {
         w4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.w + row + e) + f);
         if (MOM) m4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.m + row + e) + f);
-        if (MERGE != 0) a4[j][f] = __ldg(reinterpret_cast<const float4 *>(p.mean + e) + f);
+        if (MERGE != 0) a4[j][f] = mean_of(__ldg(reinterpret_cast<const float4 *>(p.mean + e) + f), p);
         if (MERGE == 2) s4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.snap_in + row + e) + f);
       }
     }
@@ -197,8 +217,8 @@ __global__ void __launch_bounds__(kThreads) k_local_step_scalar(const Params p, 
   const float g = BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(p.g)[i])
                        : static_cast<const float *>(p.g)[i];
   step_elem<MOM>(w, m, g, p);
-  if (MERGE == 1) w = blend_xi(w, p.mean[col], p);
-  if (MERGE == 2) w = blend_delta(w, p.mean[col], p.snap_in[i]);
+  if (MERGE == 1) w = blend_xi(w, mean_of(p.mean[col], p), p);
+  if (MERGE == 2) w = blend_delta(w, mean_of(p.mean[col], p), p.snap_in[i]);
   p.w_out[i] = w;
   if (MOM) p.m[i] = m;
   if (SNAP) p.snap_out[i] = w;
@@ -281,8 +301,8 @@ __global__ void __launch_bounds__(kThreads) k_reduce_vec(const Params p) {
     add4(acc[c][2], acc[c][3]);
     add4(acc[c][0], acc[c][2]);
     float4 r;
-    r.x = __fdiv_rn(acc[c][0].x, kf); r.y = __fdiv_rn(acc[c][0].y, kf);
-    r.z = __fdiv_rn(acc[c][0].z, kf); r.w = __fdiv_rn(acc[c][0].w, kf);
+    r.x = finish_mean(acc[c][0].x, kf, p); r.y = finish_mean(acc[c][0].y, kf, p);
+    r.z = finish_mean(acc[c][0].z, kf, p); r.w = finish_mean(acc[c][0].w, kf, p);
     reinterpret_cast<float4 *>(p.mean_out)[u] = r;  // re-read by the merge: leave it cacheable
   }
 }
@@ -312,8 +332,8 @@ __global__ void __launch_bounds__(kThreads) k_reduce_small(const Params p) {
     add4(v[c][2], v[c][3]);
     add4(v[c][0], v[c][2]);
     float4 r;
-    r.x = __fdiv_rn(v[c][0].x, kf); r.y = __fdiv_rn(v[c][0].y, kf);
-    r.z = __fdiv_rn(v[c][0].z, kf); r.w = __fdiv_rn(v[c][0].w, kf);
+    r.x = finish_mean(v[c][0].x, kf, p); r.y = finish_mean(v[c][0].y, kf, p);
+    r.z = finish_mean(v[c][0].z, kf, p); r.w = finish_mean(v[c][0].w, kf, p);
     reinterpret_cast<float4 *>(p.mean_out)[u] = r;
   }
 }
@@ -324,7 +344,7 @@ __global__ void __launch_bounds__(kThreads) k_reduce_scalar(const Params p, long
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   for (int k = 0; k < p.K; ++k) acc[k & 3] = __fadd_rn(acc[k & 3], p.snap_in[(long long)k * p.ld + col]);
   const float s = __fadd_rn(__fadd_rn(acc[0], acc[1]), __fadd_rn(acc[2], acc[3]));
-  p.mean_out[col] = __fdiv_rn(s, (float)p.K);
+  p.mean_out[col] = finish_mean(s, (float)p.K, p);
 }
 
 // ---------------------------------------------------------------- delayed merge
@@ -341,7 +361,7 @@ __global__ void __launch_bounds__(kThreads) k_merge_vec(const Params p) {
   const long long e = u * EPU;
   float4 a[F4];
 #pragma unroll
-  for (int f = 0; f < F4; ++f) a[f] = __ldg(reinterpret_cast<const float4 *>(p.mean + e) + f);
+  for (int f = 0; f < F4; ++f) a[f] = mean_of(__ldg(reinterpret_cast<const float4 *>(p.mean + e) + f), p);
   for (int k0 = 0; k0 < p.K; k0 += KB) {
     float4 w[KB][F4], s[KB][F4];
 #pragma unroll
@@ -389,7 +409,7 @@ template <bool BF16, int MODE, bool SNAP>
 __global__ void __launch_bounds__(kThreads) k_merge_scalar(const Params p, long long p0) {
   const long long col = p0 + (long long)blockIdx.x * kThreads + threadIdx.x;
   if (col >= p.P) return;
-  const float a = p.mean[col];
+  const float a = mean_of(p.mean[col], p);
   for (int k = 0; k < p.K; ++k) {
     const long long i = (long long)k * p.ld + col;
     float w = p.w[i];
