@@ -262,12 +262,16 @@ def run_reference(args, wl, name):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(wl, name, sched):
+def workload_config(wl, name, sched, shard="replicas", world=1):
     cfg = {"workload": f"{name}: K={wl['K']} replicas x P={wl['P']} {'bf16 gradients + f32 master' if wl.get('bf16') else 'float32'}, momentum {wl['momentum']}, "
                        f"weight decay {wl['weight_decay']}, lr {wl['lr']}, tau={wl['tau']}, d={wl['d']}, xi={wl['xi']}",
            "K": wl["K"], "P": wl["P"], "tau": wl["tau"], "d": wl["d"], "xi": wl["xi"],
            "l2_policy": "inputs larger than L2 (every step streams all K*P-sized arrays; gradients come from a ring of buffers)",
            "parallelism": "independent replicas of the workload per GPU (no collective on this path)"}
+    if shard == "workers":
+        cfg["parallelism"] = (f"worker axis sharded: {wl['K']} of {wl['K'] * world} workers per GPU; one ncclAllReduce of the "
+                              "partial sums (P float32) per snapshot on the side stream")
+        cfg["K_total"] = wl["K"] * world
     if sched is not None:
         cfg["schedule"] = sched
     return cfg
@@ -303,8 +307,23 @@ class Bench:
         self.dist = None
         if self.world > 1 or args.force_dist:
             import torch.distributed as dist
+            if "RANK" not in os.environ:     # a single rank started without a launcher
+                os.environ.update(RANK="0", WORLD_SIZE="1", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1",
+                                  MASTER_PORT=str(_free_port()))
             dist.init_process_group("nccl", device_id=torch.device("cuda", self.local_rank))
             self.dist = dist
+        # --shard workers: the K workers of every rank are shards of one K*world-worker job; the partial sums
+        # are exchanged by the library's own NCCL communicator (rank 0 makes the id, torch broadcasts it)
+        self.comm = None
+        if args.shard == "workers":
+            uid = torch.zeros(128, dtype=torch.uint8)
+            if self.rank == 0:
+                uid = torch.frombuffer(bytearray(B.dasgd_nccl_unique_id()), dtype=torch.uint8).clone()
+            if self.dist is not None:
+                dev = uid.cuda()
+                self.dist.broadcast(dev, 0)
+                uid = dev.cpu()
+            self.comm = B.dasgd_nccl_comm_init(bytes(uid.numpy().tobytes()), self.world, self.rank, self.local_rank)
 
     def barrier(self):
         if self.dist is not None:
@@ -328,7 +347,11 @@ class Bench:
                     dtype=B.DASGD_BF16_MASTER_F32 if wl.get("bf16") else B.DASGD_F32,
                     n_chunks=sched["n_chunks"] if flags is None else 0, device=self.local_rank,
                     host_staging=host_staging, order_after_current=False, snapshot_arrays=snapshot_arrays)
-        e.set_state(inputs.shared_start(1000 + self.rank, wl["P"], wl["w_std"], device="cuda"))
+        if self.comm is not None and not (e.cfg.flags & B.DASGD_FLAG_INLINE_MEAN):
+            e.set_shard(wl["K"] * self.world, nccl_comm=self.comm)
+        # independent replicas: every rank its own start; shards of one job: the common start of all workers
+        seed = 1000 if self.comm is not None else 1000 + self.rank
+        e.set_state(inputs.shared_start(seed, wl["P"], wl["w_std"], device="cuda"))
         return e
 
     def timed(self, e, steps, step_fn, t0=0):
@@ -482,7 +505,7 @@ def run_ours(args, wl, name, bench=None, compact=False):
 
     # ---- ablation: the same work with the mean computed inside the step kernel (no side stream)
     ablation = None
-    if not args.no_ablation:
+    if not args.no_ablation and bench.comm is None:
         eng = bench.make(wl, sched, flags=B.DASGD_FLAG_INLINE_MEAN, snapshot_arrays=False)
         a = bench.repeated(eng, args.steps, args.warmup, min(3, args.repeats), dev_step)
         bytes_a = (step_bytes(wl) * wl["tau"] + 8.0 / K) / wl["tau"]
@@ -541,7 +564,7 @@ def run_ours(args, wl, name, bench=None, compact=False):
         "ms_per_step": ms, "ms_per_step_min": m["headline"]["min"], "ms_per_step_max": m["headline"]["max"],
         "repeats": args.repeats, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 gradients, f32 state" if bf16 else "f32", "data": "synthetic",
-        "config": workload_config(wl, name, sched),
+        "config": workload_config(wl, name, sched, args.shard, world),
         "clocks": clocks, "e2e": e2e, "gpu_launches": m["headline"]["launches"],
         "roofline": {"bound": "hbm", "kernel": kname,
                      "achieved": step_gbs, "peak": peak, "unit": "GB/s",
@@ -747,6 +770,9 @@ def main():
     ap.add_argument("--chunks", type=int, default=0,
                     help="column ranges of the d = 1 pipeline (merge folded into the step kernel); 0: by size "
                          "(ranges of about 24 MiB of weights); 1: off (separate merge kernel)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "workers"],
+                    help="replicas: every GPU runs its own copy of the workload (default).  workers: the K workers of "
+                         "every GPU are shards of one K*N-worker job; the partial sums are all-reduced over NCCL")
     ap.add_argument("--sweep", action="store_true", help="run the K x tau x d sweep instead (one JSON line per point)")
     args = ap.parse_args()
     if args.warmup < 3:
