@@ -1,9 +1,12 @@
 """The five benchmark configurations at full size, in the launch configuration bench.py times
-(both fusion flags on), checked against the CPU oracle.
+(rotating snapshots, merge folded into the step kernel: chunked pipeline with two lanes when d = 1),
+checked against the CPU oracle.
 
 Every operation of the path is independent across the parameter index p, so the oracle runs on a
-sample of columns (the first and last tile of each row plus random ones) with gradients regenerated
-on the host by the same counter-based generator; the GPU works on the full arrays.
+sample of columns -- at least one from EVERY 4096-column tile of the vector kernels, the first and last
+tile of each row in full, plus random ones -- with gradients regenerated on the host by the same
+counter-based generator; the GPU works on the full arrays.  Configuration 2 is also compared on every one of
+its K*P elements.
 """
 import numpy as np
 import pytest
@@ -14,7 +17,12 @@ from paper_2006_00441_b200 import inputs
 from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, to_oracle_grad
 
 pytestmark = pytest.mark.gpu
-FUSED = 0x4 | 0x8   # merge folded into the step kernel when d >= 2; snapshots by array rotation
+FUSED = 0x4 | 0x8 | 0x100   # snapshots by array rotation; merge folded into the step kernel; two lanes when chunked
+CHUNK_BYTES = 24 << 20      # the benchmark's policy: column ranges of about 24 MiB of the weight array
+
+
+def chunks_for(K, P, d):
+    return max(2, min(1024, round(K * P * 4 / CHUNK_BYTES))) if d == 1 and P >= 2 * 4096 else 0
 
 
 @pytest.fixture(scope="module")
@@ -23,18 +31,28 @@ def B():
     return binding
 
 
-def sample_columns(P, n_random=6000, edge=4096 + 24, seed=0):
+def sample_columns(P, n_random=6000, edge=4096 + 24, seed=0, tile=4096):
+    """First and last `edge` columns, one column at a random offset inside every tile, and random ones."""
     r = np.random.default_rng(seed)
-    cols = set(range(min(edge, P))) | set(range(max(0, P - edge), P))
-    cols |= set(int(c) for c in r.integers(0, P, size=n_random))
-    return np.array(sorted(cols), dtype=np.int64)
+    parts = [np.arange(min(edge, P)), np.arange(max(0, P - edge), P), r.integers(0, P, size=n_random)]
+    starts = np.arange(0, P, tile, dtype=np.int64)
+    parts.append(np.minimum(starts + r.integers(0, tile, size=starts.size), P - 1))
+    return np.unique(np.concatenate(parts).astype(np.int64))
+
+
+def test_sample_columns_touch_every_tile():
+    for P in (25_600_000, 335_000_000, 4 * 4096 * 4096, 9000):
+        idx = sample_columns(P, seed=P % 97)
+        assert np.array_equal(np.unique(idx // 4096), np.arange((P + 4095) // 4096))
+        assert idx[0] == 0 and idx[-1] == P - 1
 
 
 def run_sampled(B, K, P, tau, d, xi, mom, wd, lr, T, g_std, dtype=0, ring=4, seed=0, checkpoints=(100,), flags=FUSED):
     """Full-size GPU run against the oracle on sampled columns.  Gradients: a ring of `ring` blocks."""
     gd = torch.bfloat16 if dtype else torch.float32
     idx = sample_columns(P, seed=seed)
-    gpu = B.DaSGD(K, P, tau, d, xi, mom, wd, dtype=dtype, flags=flags, order_after_current=False)
+    gpu = B.DaSGD(K, P, tau, d, xi, mom, wd, dtype=dtype, flags=flags, order_after_current=False,
+                  n_chunks=chunks_for(K, P, d) if flags & 0x4 and flags & 0x8 else 0)
     gpu.set_state(inputs.shared_start(seed, P, 0.02, device="cuda"))
     cpu = OracleDaSGD(K, len(idx), tau, d, xi, mom, wd, dtype=dtype)
     cpu.set_state(inputs.shared_start(seed, P, 0.02, p_index=idx).numpy())
@@ -119,6 +137,33 @@ def test_config2_resnet50_sized_200_steps(B):
                 checkpoints=(1, 2, 100))
 
 
+def test_config2_every_element_20_steps(B):
+    """All K*P = 204.8M elements against the OpenMP build of the oracle (the same source as the plain build),
+    in the launch configuration the benchmark times.  The gradients are the seeded generator's, made once on
+    the device and copied to the host, so both sides read the same numbers."""
+    K, P, tau, d, xi, mom, wd, lr, T = 8, 25_600_000, 1, 1, 0.25, 0.9, 1e-4, 0.1, 20
+    ring = 3
+    gpu = B.DaSGD(K, P, tau, d, xi, mom, wd, flags=FUSED, n_chunks=chunks_for(K, P, d), order_after_current=False)
+    w0 = inputs.shared_start(7, P, 0.02, device="cuda")
+    gpu.set_state(w0)
+    cpu = OracleDaSGD(K, P, tau, d, xi, mom, wd, omp=True)
+    cpu.set_state(w0.cpu().numpy())
+    dev_ring = [inputs.grad_block(7, r, K, P, 1e-3 ** 0.5, device="cuda") for r in range(ring)]
+    host_ring = [g.cpu().numpy() for g in dev_ring]
+    torch.cuda.synchronize()
+    for t in range(T):
+        gpu.step(dev_ring[t % ring], lr)
+        cpu.step(host_ring[t % ring], lr)
+        if t + 1 in (1, 2, T):
+            gpu.sync()
+            tol = TOL_STEP if t == 0 else TOL_RUN      # the first step starts from identical states
+            assert_close(gpu.w.cpu().numpy(), cpu.w, tol, f"all elements of w after {t + 1} steps")
+            assert_close(gpu.m.cpu().numpy(), cpu.m, tol, f"all elements of m after {t + 1} steps")
+    assert gpu.n_pending == cpu.n_pending == 1
+    assert_close(gpu.pending_mean(0).cpu().numpy(), cpu.pending(0)[2], TOL_RUN, "pending mean, all elements")
+    gpu.close()
+
+
 def test_config2_inline_mean_schedule(B):
     run_sampled(B, K=8, P=25_600_000, tau=1, d=1, xi=0.25, mom=0.9, wd=1e-4, lr=0.1, T=100, g_std=1e-3 ** 0.5,
                 flags=0x10)
@@ -192,7 +237,7 @@ def test_config5_mlp_full_size_500_steps(B):
     P = net.P
     idx = sample_columns(P, n_random=3000, seed=5)
     tidx = torch.from_numpy(idx).cuda()
-    gpu = B.DaSGD(K, P, tau, d, xi, 0.9, 0.0, dtype=1, flags=FUSED)
+    gpu = B.DaSGD(K, P, tau, d, xi, 0.9, 0.0, dtype=1, flags=FUSED | 0x80)   # forward/backward is the mean's window
     cpu = OracleDaSGD(K, len(idx), tau, d, xi, 0.9, 0.0, dtype=1)
     w0 = net.student_init()
     gpu.set_state(w0); cpu.set_state(w0[tidx].cpu().numpy())
