@@ -88,8 +88,9 @@ struct dasgd_ctx {
   // DASGD_FLAG_TWO_LANES: odd column ranges run on this stream, forked from and joined to the main
   // stream inside every chunked iteration, so that the kernel of range i+1 fills the SMs as the kernel
   // of range i drains instead of waiting for the stream's next command.
-  cudaStream_t s_lane = nullptr;
-  cudaEvent_t e_fork = nullptr, e_join = nullptr;
+  std::vector<cudaStream_t> lanes;      // extra lanes (lane 0 is the main stream)
+  std::vector<cudaEvent_t> e_joins;     // one per extra lane
+  cudaEvent_t e_fork = nullptr;
   // Sharded worker axis: this context holds cfg.K of K_total workers; `exchange` adds the partial sums of
   // all shards (an all-reduce) on the side stream.  0 / NULL: every worker is here.
   int32_t K_total = 0;
@@ -336,10 +337,12 @@ dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
   if (c->vec) {
     const long long units = p.P / 4;
     if (units > 0) {
-      if (p.K >= 8) dasgd::k_reduce_vec<1><<<blocks_for(units, kThreads), kThreads, 0, c->s1>>>(p);
-      else if (p.K > 4) dasgd::k_reduce_vec<2><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
-      else if (p.K > 2) dasgd::k_reduce_small<2><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
-      else dasgd::k_reduce_small<4><<<blocks_for(units, kThreads * 4), kThreads, 0, c->s1>>>(p);
+      // Shapes chosen by timing each kernel alone on B200 at P = 25.6M (fraction of the measured copy
+      // bandwidth): two columns per thread, four rows per batch, three CTAs per SM: 0.97 at K = 8,
+      // 1.02 at K = 16, 1.05 at K = 32; all rows in registers for K <= 4: 0.90 (K = 2) to 0.95 (K = 4).
+      if (p.K > 4) dasgd::k_reduce_vec<2, 4, 3><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
+      else if (p.K > 2) dasgd::k_reduce_small<2, 1><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
+      else dasgd::k_reduce_small<4, 1><<<blocks_for(units, kThreads * 4), kThreads, 0, c->s1>>>(p);
       c->launches++;
     }
     done = units * 4;
@@ -698,10 +701,17 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   }
   if (ctx->chunks > 1 && (c.flags & DASGD_FLAG_TWO_LANES)) {
     int prio = 0;
+    const int extra = 1;  // two lanes; three and four were measured and bring nothing
     bool ok = cudaStreamGetPriority(ctx->s0, &prio) == cudaSuccess &&
-              cudaStreamCreateWithPriority(&ctx->s_lane, cudaStreamNonBlocking, prio) == cudaSuccess &&
-              cudaEventCreateWithFlags(&ctx->e_fork, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&ctx->e_join, cudaEventDisableTiming) == cudaSuccess;
+              cudaEventCreateWithFlags(&ctx->e_fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < extra; ++i) {
+      cudaStream_t st = nullptr;
+      cudaEvent_t ev = nullptr;
+      ok = cudaStreamCreateWithPriority(&st, cudaStreamNonBlocking, prio) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+      if (st) ctx->lanes.push_back(st);
+      if (ev) ctx->e_joins.push_back(ev);
+    }
     if (!ok) {
       cudaGetLastError();
       dasgd_destroy(ctx);
@@ -738,12 +748,12 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
     cudaStreamSynchronize(ctx->s_copy);
     cudaStreamDestroy(ctx->s_copy);
   }
-  if (ctx->s_lane) {
-    cudaStreamSynchronize(ctx->s_lane);
-    cudaStreamDestroy(ctx->s_lane);
+  for (cudaStream_t st : ctx->lanes) {
+    cudaStreamSynchronize(st);
+    cudaStreamDestroy(st);
   }
+  for (cudaEvent_t ev : ctx->e_joins) cudaEventDestroy(ev);
   if (ctx->e_fork) cudaEventDestroy(ctx->e_fork);
-  if (ctx->e_join) cudaEventDestroy(ctx->e_join);
   for (cudaEvent_t e : ctx->e_copied) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->e_consumed) if (e) cudaEventDestroy(e);
   delete ctx;
@@ -913,14 +923,15 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
   // The mean of a range reads the weights its step kernel has just written: store them with the default
   // cache policy so that part of them is still in L2 then (everything else streams through).
   p.keep_w = s_due ? 1 : 0;
-  if (c->s_lane) {  // fork: the second lane starts after everything the main stream holds so far
+  const int n_lanes = 1 + (int)c->lanes.size();
+  if (n_lanes > 1) {  // fork: the other lanes start after everything the main stream holds so far
     CU(c, cudaEventRecord(c->e_fork, c->s0));
-    CU(c, cudaStreamWaitEvent(c->s_lane, c->e_fork, 0));
+    for (cudaStream_t st : c->lanes) CU(c, cudaStreamWaitEvent(st, c->e_fork, 0));
   }
   for (int i = 0; i < c->chunks; ++i) {
     const long long col0 = (long long)i * c->chunk_cols;
     const long long len = c->cfg.P - col0 < c->chunk_cols ? c->cfg.P - col0 : c->chunk_cols;
-    cudaStream_t lane = (c->s_lane && (i & 1)) ? c->s_lane : c->s0;
+    cudaStream_t lane = (i % n_lanes) ? c->lanes[i % n_lanes - 1] : c->s0;
     if (per_chunk_wait) {
       stall_about_to_wait(c, c->slots[ms].stall_sp_c[i], lane);
       CU(c, cudaStreamWaitEvent(lane, c->slots[ms].e_avg_c[i], 0));
@@ -937,9 +948,9 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
       sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
     }
   }
-  if (c->s_lane) {  // join: what the caller puts on the main stream next comes after both lanes
-    CU(c, cudaEventRecord(c->e_join, c->s_lane));
-    CU(c, cudaStreamWaitEvent(c->s0, c->e_join, 0));
+  for (size_t j = 0; j < c->lanes.size(); ++j) {  // join: what the caller puts on the main stream next comes after all lanes
+    CU(c, cudaEventRecord(c->e_joins[j], c->lanes[j]));
+    CU(c, cudaStreamWaitEvent(c->s0, c->e_joins[j], 0));
   }
   c->cur = out;
   c->t += 1;
@@ -1089,7 +1100,7 @@ dasgd_status dasgd_sync(dasgd_ctx *ctx) {
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(ctx->cfg.sync_timeout_ms);
   std::vector<cudaStream_t> streams = {ctx->s0, ctx->s1};
   if (ctx->s_copy) streams.push_back(ctx->s_copy);
-  if (ctx->s_lane) streams.push_back(ctx->s_lane);
+  for (cudaStream_t st : ctx->lanes) streams.push_back(st);
   for (cudaStream_t s : streams) {
     for (;;) {
       cudaError_t e = cudaStreamQuery(s);

@@ -265,9 +265,8 @@ __device__ __forceinline__ void add4(float4 &a, const float4 &b) {
 
 // U units per thread (columns u, u + kThreads, ...): with few rows more columns per thread keep
 // enough loads in flight (K = 2 ran at half the bandwidth with one column per thread).
-template <int U>
-__global__ void __launch_bounds__(kThreads) k_reduce_vec(const Params p) {
-  constexpr int KC = U == 1 ? 8 : 4;  // rows per batch of loads (a multiple of 4, so k mod 4 == j mod 4)
+template <int U, int KC /* rows per batch of loads: a multiple of 4, so k mod 4 == j mod 4 */, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) k_reduce_vec(const Params p) {
   const long long units = p.P / 4;
   const long long u0 = (long long)blockIdx.x * (kThreads * U) + threadIdx.x;
   const float4 *base = reinterpret_cast<const float4 *>(p.snap_in);
@@ -309,8 +308,8 @@ __global__ void __launch_bounds__(kThreads) k_reduce_vec(const Params p) {
 
 // K <= 4: the whole column fits in registers.  Missing rows count as +0, which leaves the pairwise
 // tree (r0 + r1) + (r2 + r3) equal to what the general kernel computes.
-template <int U>
-__global__ void __launch_bounds__(kThreads) k_reduce_small(const Params p) {
+template <int U, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) k_reduce_small(const Params p) {
   const long long units = p.P / 4;
   const long long u0 = (long long)blockIdx.x * (kThreads * U) + threadIdx.x;
   const float4 *base = reinterpret_cast<const float4 *>(p.snap_in);
