@@ -70,7 +70,7 @@ def schedule_of(wl, args):
         return {"merge": "fused", "n_chunks": 0, "lanes": 0}
     if wl["d"] == 1 and args.chunks != 1 and wl["P"] >= 2 * 4096:
         n = args.chunks if args.chunks > 0 else auto_chunks(wl["K"], wl["P"])
-        return {"merge": "chunked", "n_chunks": n, "lanes": 1 if args.lanes else 0}
+        return {"merge": "chunked", "n_chunks": n, "lanes": 1 if args.lanes else 0, "graph": 1 if args.graph else 0}
     return {"merge": "separate", "n_chunks": 0, "lanes": 0}
 
 
@@ -338,6 +338,8 @@ class Bench:
             f = B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE
         if sched.get("lanes"):
             f |= B.DASGD_FLAG_TWO_LANES
+        if sched.get("graph"):
+            f |= B.DASGD_FLAG_GRAPH
         return f | (B.DASGD_FLAG_TIMING if timing else 0)
 
     def make(self, wl, sched, timing=False, host_staging=False, flags=None, snapshot_arrays=True):
@@ -767,6 +769,7 @@ def main():
                     help="initialise the NCCL process group even with one rank (exercises the multi-rank plumbing)")
     ap.add_argument("--no-ablation", action="store_true", help="skip the inline-mean ablation leg")
     ap.add_argument("--lanes", type=int, default=1, help="1: alternate the column ranges between two streams; 0: one stream")
+    ap.add_argument("--graph", type=int, default=0, help="1: replay each chunked iteration from a CUDA graph")
     ap.add_argument("--chunks", type=int, default=0,
                     help="column ranges of the d = 1 pipeline (merge folded into the step kernel); 0: by size "
                          "(ranges of about 24 MiB of weights); 1: off (separate merge kernel)")

@@ -95,6 +95,17 @@ typedef enum {
                                          main stream before / after the call is still ordered before / after all
                                          of it.  Results are unchanged.                                        */
 
+#define DASGD_FLAG_GRAPH 0x200u        /* with n_chunks > 1: every chunked iteration is recorded once as a CUDA graph
+                                         (stream capture of the very launches the library would issue) and then
+                                         replayed, which removes most of the host's per-launch cost and lets more,
+                                         smaller column ranges pay off.  The recorded kernels read the gradients
+                                         pointer and the learning rate from a 16-byte device block that the library
+                                         allocates at dasgd_init and frees at dasgd_destroy (its only device
+                                         allocation).  A replay finishes when its last mean is complete, so the
+                                         means of one iteration overlap the step kernels of the SAME iteration only.
+                                         Ignored with DASGD_FLAG_TIMING (which times the same dependency structure
+                                         with direct launches) and with a sharded worker axis.  Results unchanged. */
+
 /* Variants of the local step.  Section IV-A states only the values of momentum and weight decay used on the
  * paper's platform and gives no formula, so the common forms are all offered; the default is the plain one. */
 #define DASGD_FLAG_NESTEROV 0x20u      /* w <- w - lr*(g' + mu*m) with the freshly updated m (needs momentum > 0) */

@@ -50,6 +50,22 @@ struct Span {
   long long units = 0;          // replica-parameters the timed launch processes
 };
 
+// One recorded iteration of the chunked pipeline: every pointer and switch that the launches depend on
+// (the gradients and the learning rate come from device memory, so they are not part of the key).
+struct GraphKey {
+  const void *w, *w_out, *mean, *snap_in, *red_in, *mean_out;
+  int mode, vec, s_due, keep_w;
+  bool operator==(const GraphKey &o) const {
+    return w == o.w && w_out == o.w_out && mean == o.mean && snap_in == o.snap_in && red_in == o.red_in &&
+           mean_out == o.mean_out && mode == o.mode && vec == o.vec && s_due == o.s_due && keep_w == o.keep_w;
+  }
+};
+struct GraphEntry {
+  GraphKey key;
+  cudaGraphExec_t exec = nullptr;
+  int64_t kernels = 0;  // kernel launches one replay stands for
+};
+
 struct DeviceGuard {
   int prev = -1;
   bool switched = false;
@@ -91,6 +107,12 @@ struct dasgd_ctx {
   std::vector<cudaStream_t> lanes;      // extra lanes (lane 0 is the main stream)
   std::vector<cudaEvent_t> e_joins;     // one per extra lane
   cudaEvent_t e_fork = nullptr;
+  // DASGD_FLAG_GRAPH: recorded iterations of the chunked pipeline, their capture-only events and the
+  // device block the replayed kernels read the gradients pointer and the learning rate from.
+  bool use_graph = false;
+  dasgd::DynArgs *dyn_dev = nullptr;
+  std::vector<GraphEntry> graphs;
+  std::vector<cudaEvent_t> cap_ev;  // per column range, then one per extra lane, then fork and side-stream join
   // Sharded worker axis: this context holds cfg.K of K_total workers; `exchange` adds the partial sums of
   // all shards (an all-reduce) on the side stream.  0 / NULL: every worker is here.
   int32_t K_total = 0;
@@ -165,7 +187,8 @@ Params columns(const dasgd_ctx *c, Params p, long long col0, long long len) {
   p.w += col0;
   p.w_out += col0;
   if (p.m) p.m += col0;
-  if (p.g) p.g = static_cast<const char *>(p.g) + (size_t)col0 * gsz;
+  if (p.dyn) p.g_off += col0;
+  else if (p.g) p.g = static_cast<const char *>(p.g) + (size_t)col0 * gsz;
   if (p.w_lp) p.w_lp += col0;
   if (p.snap_out) p.snap_out += col0;
   if (p.snap_in) p.snap_in += col0;
@@ -718,6 +741,21 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
       return fail(nullptr, DASGD_ERR_CUDA, "init: cannot create the second lane's stream and events");
     }
   }
+  if (ctx->chunks > 1 && (c.flags & DASGD_FLAG_GRAPH)) {
+    bool ok = cudaMalloc(&ctx->dyn_dev, sizeof(dasgd::DynArgs)) == cudaSuccess;
+    const size_t n_ev = (size_t)ctx->chunks + ctx->lanes.size() + 2;
+    for (size_t i = 0; ok && i < n_ev; ++i) {
+      cudaEvent_t ev = nullptr;
+      ok = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+      if (ev) ctx->cap_ev.push_back(ev);
+    }
+    if (!ok) {
+      cudaGetLastError();
+      dasgd_destroy(ctx);
+      return fail(nullptr, DASGD_ERR_CUDA, "init: cannot create the replay's device block and events");
+    }
+    ctx->use_graph = true;
+  }
   if (c.n_stage > 0) {
     bool ok = cudaStreamCreateWithFlags(&ctx->s_copy, cudaStreamNonBlocking) == cudaSuccess;
     ctx->e_copied.assign(c.n_stage, nullptr);
@@ -753,6 +791,9 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
     cudaStreamDestroy(st);
   }
   for (cudaEvent_t ev : ctx->e_joins) cudaEventDestroy(ev);
+  for (GraphEntry &g : ctx->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+  for (cudaEvent_t ev : ctx->cap_ev) cudaEventDestroy(ev);
+  if (ctx->dyn_dev) cudaFree(ctx->dyn_dev);
   if (ctx->e_fork) cudaEventDestroy(ctx->e_fork);
   for (cudaEvent_t e : ctx->e_copied) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->e_consumed) if (e) cudaEventDestroy(e);
@@ -876,6 +917,92 @@ dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, 
 // stream goes on with ranges i+1, ...  The mean of range i thus has the rest of this iteration and the
 // first i ranges of the next one as its window (the condition t_c < d*t_p of Eq. 6, per range), although
 // the next iteration's kernels consume it directly.
+// The launches of one chunked iteration, enqueued on the main stream, the extra lanes and the side stream.
+// Used while a stream capture is active; `ev` are capture-only events.
+dasgd_status enqueue_chunked(dasgd_ctx *c, const Params &p, const Params &q, int mode, bool vec, bool s_due) {
+  const int n_lanes = 1 + (int)c->lanes.size();
+  cudaEvent_t *ev_chunk = c->cap_ev.data();
+  cudaEvent_t *ev_lane = ev_chunk + c->chunks;
+  cudaEvent_t ev_fork = ev_lane[c->lanes.size()], ev_side = ev_lane[c->lanes.size() + 1];
+  CU(c, cudaEventRecord(ev_fork, c->s0));
+  for (cudaStream_t st : c->lanes) CU(c, cudaStreamWaitEvent(st, ev_fork, 0));
+  for (int i = 0; i < c->chunks; ++i) {
+    const long long col0 = (long long)i * c->chunk_cols;
+    const long long len = c->cfg.P - col0 < c->chunk_cols ? c->cfg.P - col0 : c->chunk_cols;
+    cudaStream_t lane = (i % n_lanes) ? c->lanes[i % n_lanes - 1] : c->s0;
+    dasgd_status st = launch_step(c, columns(c, p, col0, len), vec, mode, false, lane);
+    if (st != DASGD_OK) return st;
+    if (s_due) {
+      CU(c, cudaEventRecord(ev_chunk[i], lane));
+      CU(c, cudaStreamWaitEvent(c->s1, ev_chunk[i], 0));
+      st = launch_mean(c, columns(c, q, col0, len));
+      if (st != DASGD_OK) return st;
+    }
+  }
+  for (size_t j = 0; j < c->lanes.size(); ++j) {
+    CU(c, cudaEventRecord(ev_lane[j], c->lanes[j]));
+    CU(c, cudaStreamWaitEvent(c->s0, ev_lane[j], 0));
+  }
+  if (s_due) {
+    CU(c, cudaEventRecord(ev_side, c->s1));
+    CU(c, cudaStreamWaitEvent(c->s0, ev_side, 0));
+  }
+  return DASGD_OK;
+}
+
+// One chunked iteration as the replay of a recorded CUDA graph (recorded on first use of a combination of
+// arrays and switches).  The recording holds the step kernels on the lanes and the means on the side stream
+// with the same dependencies as the direct launches; gradients pointer and learning rate are read from
+// device memory, written by a one-thread kernel just before the replay.  If recording fails, replay is
+// switched off for this context (c->use_graph = false) and the caller launches directly.
+dasgd_status replay_chunked(dasgd_ctx *c, Params p, const Params &q, const void *grads, float lr, int mode, bool vec,
+                            bool m_due, bool s_due, bool per_chunk_wait, int ms) {
+  if (m_due && per_chunk_wait)  // the mean that lands was made by direct launches: order after all of it
+    for (cudaEvent_t e : c->slots[ms].e_avg_c) CU(c, cudaStreamWaitEvent(c->s0, e, 0));
+  p.g = nullptr;
+  p.dyn = c->dyn_dev;
+  p.g_off = 0;
+  GraphKey key{p.w, p.w_out, p.mean, p.snap_in, q.snap_in, q.mean_out, mode, vec ? 1 : 0, s_due ? 1 : 0, p.keep_w};
+  GraphEntry *entry = nullptr;
+  for (GraphEntry &g : c->graphs)
+    if (g.key == key) { entry = &g; break; }
+  if (!entry) {
+    const int64_t launches_before = c->launches;
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamBeginCapture(c->s0, cudaStreamCaptureModeRelaxed);
+    dasgd_status st = e == cudaSuccess ? enqueue_chunked(c, p, q, mode, vec, s_due) : DASGD_ERR_CUDA;
+    if (e == cudaSuccess) {
+      e = cudaStreamEndCapture(c->s0, &graph);  // always ends the capture, also after a failed launch
+      if (st == DASGD_OK && e != cudaSuccess) st = DASGD_ERR_CUDA;
+    }
+    cudaGraphExec_t exec = nullptr;
+    if (st == DASGD_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) st = DASGD_ERR_CUDA;
+    if (graph) cudaGraphDestroy(graph);
+    const int64_t kernels = c->launches - launches_before;
+    c->launches = launches_before;
+    if (st != DASGD_OK) {
+      cudaGetLastError();
+      c->use_graph = false;
+      return DASGD_OK;
+    }
+    if (c->graphs.size() >= 64) {  // the combinations of a run are few; a long list means something cycles
+      cudaGraphExecDestroy(c->graphs.front().exec);
+      c->graphs.erase(c->graphs.begin());
+    }
+    GraphEntry ge;
+    ge.key = key;
+    ge.exec = exec;
+    ge.kernels = kernels;
+    c->graphs.push_back(ge);
+    entry = &c->graphs.back();
+  }
+  dasgd::k_set_dyn<<<1, 1, 0, c->s0>>>(c->dyn_dev, grads, lr);
+  CU(c, cudaGetLastError());
+  CU(c, cudaGraphLaunch(entry->exec, c->s0));
+  c->launches += entry->kernels + 1;
+  return DASGD_OK;
+}
+
 dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due, bool s_due) {
   Params p = base_params(c);
   p.g = grads;
@@ -923,6 +1050,27 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
   // The mean of a range reads the weights its step kernel has just written: store them with the default
   // cache policy so that part of them is still in L2 then (everything else streams through).
   p.keep_w = s_due ? 1 : 0;
+  if (c->use_graph && !(c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0) {
+    dasgd_status gst = replay_chunked(c, p, q, grads, lr, mode, vec, m_due, s_due, per_chunk_wait, ms);
+    if (gst != DASGD_OK) return gst;
+    if (c->use_graph) {  // replayed (a failed capture switches replay off and falls through to direct launches)
+      c->cur = out;
+      c->t += 1;
+      if (m_due) release_oldest(c);
+      if (s_due) {
+        Slot &sl = c->slots[ns];
+        CU(c, cudaEventRecord(sl.e_avg, c->s0));  // the replay is complete on the main stream: so is the mean
+        sl.state = SLOT_AVERAGING;
+        sl.chunked = false;
+        sl.s = c->t;
+        sl.buf = out;
+        c->frozen[out] += 1;
+        sl.holds = true;
+        c->pending.push_back(ns);
+      }
+      return DASGD_OK;
+    }
+  }
   const int n_lanes = 1 + (int)c->lanes.size();
   if (n_lanes > 1) {  // fork: the other lanes start after everything the main stream holds so far
     CU(c, cudaEventRecord(c->e_fork, c->s0));
@@ -947,6 +1095,13 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
       CU(c, cudaEventRecord(sl.e_avg_c[i], c->s1));
       sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
     }
+  }
+  if (c->use_graph && (c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0 && s_due) {
+    // Timing pass of the replayed schedule: a replay ends only when its last mean is complete, so the
+    // main stream waits for it here as well (and that wait is accounted as stall like any other).
+    Slot &sl = c->slots[ns];
+    stall_about_to_wait(c, sl.stall_sp_c[c->chunks - 1], c->s0);
+    CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg_c[c->chunks - 1], 0));
   }
   for (size_t j = 0; j < c->lanes.size(); ++j) {  // join: what the caller puts on the main stream next comes after all lanes
     CU(c, cudaEventRecord(c->e_joins[j], c->lanes[j]));

@@ -28,6 +28,14 @@ namespace dasgd {
 
 constexpr int kThreads = 256;
 
+// Arguments that change from one iteration to the next, kept in device memory so that a launch recorded
+// once (CUDA graph) can be replayed with new values.
+struct DynArgs {
+  const void *g;  // [K][ld] gradients of this iteration
+  float lr;
+  int pad;
+};
+
 struct Params {
   const float *w;       // [K][ld] weights to read
   float *w_out;         // [K][ld] where the new weights go (== w for an in-place update)
@@ -43,6 +51,8 @@ struct Params {
   float lr, mu, lambda, xi, omx;
   int nesterov;      // 1: step along g' + mu*m instead of m
   int decoupled_wd;  // 1: weight decay is applied to the weights directly, not added to the gradient
+  const DynArgs *dyn;  // non-NULL: take g and lr from there (g_off = first column of this launch)
+  long long g_off;
   float mean_div;    // 0: `mean` holds the mean.  Otherwise `mean` holds the SUM over all workers (sharded
                      //    worker axis) and the mean is that sum divided, correctly rounded, by this number
   int sum_only;      // 1: the worker-axis kernel writes the plain sum of its K rows, not their mean
@@ -68,7 +78,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // ---------------------------------------------------------------- scalar arithmetic
 
 template <bool MOM>
-__device__ __forceinline__ void step_elem(float &w, float &m, float g, const Params &p) {
+__device__ __forceinline__ void step_elem(float &w, float &m, float g, const Params &p, float lr) {
   // the two variant switches are uniform across the grid, so the branches cost nothing here
   const float gp = p.decoupled_wd ? g : fmaf(p.lambda, w, g);
   float dir = gp;
@@ -77,8 +87,8 @@ __device__ __forceinline__ void step_elem(float &w, float &m, float g, const Par
     dir = p.nesterov ? fmaf(p.mu, m, gp) : m;
   }
   const float w_old = w;
-  w = fmaf(-p.lr, dir, w);
-  if (p.decoupled_wd) w = fmaf(-__fmul_rn(p.lr, p.lambda), w_old, w);
+  w = fmaf(-lr, dir, w);
+  if (p.decoupled_wd) w = fmaf(-__fmul_rn(lr, p.lambda), w_old, w);
 }
 
 // The mean as the merge sees it: stored as such, or formed here from the all-worker sum.
@@ -136,6 +146,12 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
   }
   const long long row = (long long)k * p.ld;
   const long long u0 = tile * (long long)(kThreads * UNROLL) + threadIdx.x;
+  const void *gbase = p.g;
+  float lr = p.lr;
+  if (p.dyn) {
+    gbase = static_cast<const char *>(p.dyn->g) + p.g_off * (BF16 ? 2 : 4);
+    lr = p.dyn->lr;
+  }
 
   float4 w4[UNROLL][F4], m4[UNROLL][F4], g4[UNROLL][F4], a4[UNROLL][F4], s4[UNROLL][F4];
   bool ok[UNROLL];
@@ -147,13 +163,13 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
     if (ok[j]) {
       const long long e = u * EPU;  // element offset inside the row
       if (BF16) {
-        const uint4 gb = ld_stream(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.g) + row + e));
+        const uint4 gb = ld_stream(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(gbase) + row + e));
         g4[j][0] = make_float4(bf16_bits_to_f32(gb.x & 0xFFFFu), bf16_bits_to_f32(gb.x >> 16),
                                bf16_bits_to_f32(gb.y & 0xFFFFu), bf16_bits_to_f32(gb.y >> 16));
         g4[j][F4 - 1] = make_float4(bf16_bits_to_f32(gb.z & 0xFFFFu), bf16_bits_to_f32(gb.z >> 16),
                                     bf16_bits_to_f32(gb.w & 0xFFFFu), bf16_bits_to_f32(gb.w >> 16));
       } else {
-        g4[j][0] = ld_stream(reinterpret_cast<const float4 *>(static_cast<const float *>(p.g) + row + e));
+        g4[j][0] = ld_stream(reinterpret_cast<const float4 *>(static_cast<const float *>(gbase) + row + e));
       }
 #pragma unroll
       for (int f = 0; f < F4; ++f) {
@@ -174,10 +190,10 @@ __global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
       float4 w = w4[j][f];
       float4 m = MOM ? m4[j][f] : make_float4(0.f, 0.f, 0.f, 0.f);
       const float4 g = g4[j][f];
-      step_elem<MOM>(w.x, m.x, g.x, p);
-      step_elem<MOM>(w.y, m.y, g.y, p);
-      step_elem<MOM>(w.z, m.z, g.z, p);
-      step_elem<MOM>(w.w, m.w, g.w, p);
+      step_elem<MOM>(w.x, m.x, g.x, p, lr);
+      step_elem<MOM>(w.y, m.y, g.y, p, lr);
+      step_elem<MOM>(w.z, m.z, g.z, p, lr);
+      step_elem<MOM>(w.w, m.w, g.w, p, lr);
       if (MERGE == 1) {
         const float4 a = a4[j][f];
         DASGD_F4_APPLY(w, blend_xi(w.x, a.x, p), blend_xi(w.y, a.y, p), blend_xi(w.z, a.z, p), blend_xi(w.w, a.w, p))
@@ -214,9 +230,15 @@ __global__ void __launch_bounds__(kThreads) k_local_step_scalar(const Params p, 
   if (col >= p.P) return;
   const long long i = (long long)k * p.ld + col;
   float w = p.w[i], m = MOM ? p.m[i] : 0.0f;
-  const float g = BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(p.g)[i])
-                       : static_cast<const float *>(p.g)[i];
-  step_elem<MOM>(w, m, g, p);
+  const void *gbase = p.g;
+  float lr = p.lr;
+  if (p.dyn) {
+    gbase = static_cast<const char *>(p.dyn->g) + p.g_off * (BF16 ? 2 : 4);
+    lr = p.dyn->lr;
+  }
+  const float g = BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(gbase)[i])
+                       : static_cast<const float *>(gbase)[i];
+  step_elem<MOM>(w, m, g, p, lr);
   if (MERGE == 1) w = blend_xi(w, mean_of(p.mean[col], p), p);
   if (MERGE == 2) w = blend_delta(w, mean_of(p.mean[col], p), p.snap_in[i]);
   p.w_out[i] = w;
@@ -479,10 +501,10 @@ __global__ void __launch_bounds__(kThreads) k_step_allk_vec(const Params p) {
           float4 x = w[j][f];
           float4 y = MOM ? m[j][f] : make_float4(0.f, 0.f, 0.f, 0.f);
           const float4 gg = g[j][f];
-          step_elem<MOM>(x.x, y.x, gg.x, p);
-          step_elem<MOM>(x.y, y.y, gg.y, p);
-          step_elem<MOM>(x.z, y.z, gg.z, p);
-          step_elem<MOM>(x.w, y.w, gg.w, p);
+          step_elem<MOM>(x.x, y.x, gg.x, p, p.lr);
+          step_elem<MOM>(x.y, y.y, gg.y, p, p.lr);
+          step_elem<MOM>(x.z, y.z, gg.z, p, p.lr);
+          step_elem<MOM>(x.w, y.w, gg.w, p, p.lr);
           if (MERGE) {
             DASGD_F4_APPLY(x, blend_xi(x.x, a[f].x, p), blend_xi(x.y, a[f].y, p), blend_xi(x.z, a[f].z, p),
                            blend_xi(x.w, a[f].w, p))
@@ -529,7 +551,7 @@ __global__ void __launch_bounds__(kThreads) k_step_allk_scalar(const Params p, l
     float w = p.w[i], m = MOM ? p.m[i] : 0.0f;
     const float g = BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(p.g)[i])
                          : static_cast<const float *>(p.g)[i];
-    step_elem<MOM>(w, m, g, p);
+    step_elem<MOM>(w, m, g, p, p.lr);
     if (MERGE) w = blend_xi(w, a, p);
     p.w_out[i] = w;
     if (MOM) p.m[i] = m;
@@ -538,6 +560,13 @@ __global__ void __launch_bounds__(kThreads) k_step_allk_scalar(const Params p, l
   }
   if (MEANOUT)
     p.mean_out[col] = __fdiv_rn(__fadd_rn(__fadd_rn(acc[0], acc[1]), __fadd_rn(acc[2], acc[3])), (float)p.K);
+}
+
+// ---------------------------------------------------------------- per-iteration arguments of a replayed launch
+
+__global__ void k_set_dyn(DynArgs *dyn, const void *g, float lr) {
+  dyn->g = g;
+  dyn->lr = lr;
 }
 
 // ---------------------------------------------------------------- bf16 copy of the master weights
