@@ -47,7 +47,9 @@ WORKLOADS = {
 }
 METRIC = "replica-param updates/s"
 UNIT = "updates/s"
-CHUNK_BYTES = 24 << 20   # target size of one column range of the weight array in the d = 1 pipeline
+CHUNK_BYTES = 18 << 20   # target size of one column range of the weight array in the d = 1 pipeline
+HOST_US_PER_RANGE = 16.0  # host time to enqueue one range (four CUDA calls); more ranges than the iteration has
+                          # time for would make the host the bottleneck
 
 
 def step_bytes(wl):
@@ -57,9 +59,13 @@ def step_bytes(wl):
     return 20 if wl["momentum"] else 12   # read w, (m,) g; write w (, m)
 
 
-def auto_chunks(K, P):
-    """Column ranges of the d = 1 pipeline by size: ranges of about CHUNK_BYTES of the [K][P] weight array."""
-    return max(2, min(1024, round(K * P * 4 / CHUNK_BYTES)))
+def auto_chunks(K, P, bytes_per_update=25.0):
+    """Column ranges of the d = 1 pipeline: ranges of about CHUNK_BYTES of the [K][P] weight array (small enough
+    that the mean of a range finds much of it still in L2), but no more than the host can enqueue in the time
+    the GPU needs for one iteration (estimated at the measured copy bandwidth)."""
+    by_size = round(K * P * 4 / CHUNK_BYTES)
+    iteration_us = K * P * bytes_per_update / (measured_peak_gbs()[0] * 1e9) * 1e6
+    return int(max(2, min(1024, by_size, iteration_us / HOST_US_PER_RANGE)))
 
 
 def schedule_of(wl, args):
@@ -772,7 +778,7 @@ def main():
     ap.add_argument("--graph", type=int, default=0, help="1: replay each chunked iteration from a CUDA graph")
     ap.add_argument("--chunks", type=int, default=0,
                     help="column ranges of the d = 1 pipeline (merge folded into the step kernel); 0: by size "
-                         "(ranges of about 24 MiB of weights); 1: off (separate merge kernel)")
+                         "(ranges of about 18 MiB of weights); 1: off (separate merge kernel)")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "workers"],
                     help="replicas: every GPU runs its own copy of the workload (default).  workers: the K workers of "
                          "every GPU are shards of one K*N-worker job; the partial sums are all-reduced over NCCL")

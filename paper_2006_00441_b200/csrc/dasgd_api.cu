@@ -528,11 +528,10 @@ dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
   Slot &sl = c->slots[slot];
   if (sl.state != SLOT_AVERAGING)
     return fail(c, DASGD_ERR_BAD_STATE, "merge: the oldest snapshot has not been given to dasgd_average_async");
-  if (sl.chunked) {
-    for (size_t i = 0; i < sl.e_avg_c.size(); ++i) {
-      stall_about_to_wait(c, sl.stall_sp_c[i], c->s0);
-      CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg_c[i], 0));
-    }
+  if (sl.chunked) {  // the means of the ranges run in order on the side stream: the last one implies the rest
+    const size_t last = sl.e_avg_c.size() - 1;
+    stall_about_to_wait(c, sl.stall_sp_c[last], c->s0);
+    CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg_c[last], 0));
   } else {
     stall_about_to_wait(c, sl.stall_sp, c->s0);
     CU(c, cudaStreamWaitEvent(c->s0, sl.e_avg, 0));
@@ -958,7 +957,7 @@ dasgd_status enqueue_chunked(dasgd_ctx *c, const Params &p, const Params &q, int
 dasgd_status replay_chunked(dasgd_ctx *c, Params p, const Params &q, const void *grads, float lr, int mode, bool vec,
                             bool m_due, bool s_due, bool per_chunk_wait, int ms) {
   if (m_due && per_chunk_wait)  // the mean that lands was made by direct launches: order after all of it
-    for (cudaEvent_t e : c->slots[ms].e_avg_c) CU(c, cudaStreamWaitEvent(c->s0, e, 0));
+    CU(c, cudaStreamWaitEvent(c->s0, c->slots[ms].e_avg_c.back(), 0));
   p.g = nullptr;
   p.dyn = c->dyn_dev;
   p.g_off = 0;
@@ -1076,13 +1075,24 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
     CU(c, cudaEventRecord(c->e_fork, c->s0));
     for (cudaStream_t st : c->lanes) CU(c, cudaStreamWaitEvent(st, c->e_fork, 0));
   }
-  for (int i = 0; i < c->chunks; ++i) {
+  // "Mean of range i complete" is signalled per group of G consecutive ranges (an event after the last mean of
+  // the group: the side stream runs them in order), and a lane waits once per group it enters.  A range thus
+  // waits for the means of up to G-1 later ranges of the previous iteration, all of which were started at least
+  // C-G ranges ago; with G = C/8 that costs nothing and saves most of the event calls.
+  const int C = c->chunks;
+  const int G = C >= 16 ? C / 8 : 1;
+  auto group_end = [&](int i) { const int e = (i / G + 1) * G - 1; return e < C - 1 ? e : C - 1; };
+  std::vector<int> waited(n_lanes, -1);
+  for (int i = 0; i < C; ++i) {
     const long long col0 = (long long)i * c->chunk_cols;
     const long long len = c->cfg.P - col0 < c->chunk_cols ? c->cfg.P - col0 : c->chunk_cols;
-    cudaStream_t lane = (i % n_lanes) ? c->lanes[i % n_lanes - 1] : c->s0;
-    if (per_chunk_wait) {
-      stall_about_to_wait(c, c->slots[ms].stall_sp_c[i], lane);
-      CU(c, cudaStreamWaitEvent(lane, c->slots[ms].e_avg_c[i], 0));
+    const int li = i % n_lanes;
+    cudaStream_t lane = li ? c->lanes[li - 1] : c->s0;
+    if (per_chunk_wait && waited[li] < group_end(i)) {
+      const int e = group_end(i);
+      stall_about_to_wait(c, c->slots[ms].stall_sp_c[e], lane);
+      CU(c, cudaStreamWaitEvent(lane, c->slots[ms].e_avg_c[e], 0));
+      waited[li] = e;
     }
     dasgd_status st = launch_step(c, columns(c, p, col0, len), vec, mode, false, lane);
     if (st != DASGD_OK) return st;
@@ -1092,8 +1102,10 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
       CU(c, cudaStreamWaitEvent(c->s1, sl.e_snap_c[i], 0));
       st = launch_mean(c, columns(c, q, col0, len));
       if (st != DASGD_OK) return st;
-      CU(c, cudaEventRecord(sl.e_avg_c[i], c->s1));
-      sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
+      if (i == group_end(i)) {
+        CU(c, cudaEventRecord(sl.e_avg_c[i], c->s1));
+        sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
+      }
     }
   }
   if (c->use_graph && (c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0 && s_due) {

@@ -18,11 +18,10 @@ from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, to_oracle_
 
 pytestmark = pytest.mark.gpu
 FUSED = 0x4 | 0x8 | 0x100   # snapshots by array rotation; merge folded into the step kernel; two lanes when chunked
-CHUNK_BYTES = 24 << 20      # the benchmark's policy: column ranges of about 24 MiB of the weight array
-
-
 def chunks_for(K, P, d):
-    return max(2, min(1024, round(K * P * 4 / CHUNK_BYTES))) if d == 1 and P >= 2 * 4096 else 0
+    """The benchmark's policy for the number of column ranges."""
+    import bench
+    return bench.auto_chunks(K, P) if d == 1 and P >= 2 * 4096 else 0
 
 
 @pytest.fixture(scope="module")
