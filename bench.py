@@ -48,8 +48,9 @@ WORKLOADS = {
 METRIC = "replica-param updates/s"
 UNIT = "updates/s"
 CHUNK_BYTES = 18 << 20   # target size of one column range of the weight array in the d = 1 pipeline
-HOST_US_PER_RANGE = 16.0  # host time to enqueue one range (four CUDA calls); more ranges than the iteration has
-                          # time for would make the host the bottleneck
+HOST_US_PER_RANGE = 20.0  # host time to enqueue one range (four CUDA calls, about 14 us measured) with some margin:
+                          # more ranges than the iteration has time for would make the host the bottleneck
+MIN_RANGE_COLS = 409_600  # narrower ranges leave the mean kernel too few columns to fill the GPU (K >= 16)
 
 
 def step_bytes(wl):
@@ -65,7 +66,7 @@ def auto_chunks(K, P, bytes_per_update=25.0):
     the GPU needs for one iteration (estimated at the measured copy bandwidth)."""
     by_size = round(K * P * 4 / CHUNK_BYTES)
     iteration_us = K * P * bytes_per_update / (measured_peak_gbs()[0] * 1e9) * 1e6
-    return int(max(2, min(1024, by_size, iteration_us / HOST_US_PER_RANGE)))
+    return int(max(2, min(1024, by_size, iteration_us / HOST_US_PER_RANGE, P / MIN_RANGE_COLS)))
 
 
 def schedule_of(wl, args):
