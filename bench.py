@@ -199,7 +199,7 @@ def oracle_throughput(wl, seconds_budget: float, steps: int | None = None, warmu
     cores = probe.threads
     probe.close()
     # calibrate on a slice too large for the CPU caches, so the rate is the DRAM-bound one
-    Pc = min(wl["P"], 2_000_000 if omp else 500_000)
+    Pc = min(wl["P"], 2_000_000)
     odt = 1 if wl.get("bf16") else 0
 
     def host_grad(t, idx):

@@ -8,12 +8,12 @@
  * What it follows:
  *   - Local step: Eq. 2, "otherwise" branch (Section III-C-1; restated in
  *     Appendix "Update Rule"):  x <- x - eta * g(x).  Momentum and weight decay are
- *     only named as hyper-parameters in Section IV-A ("weight decay 0.01, moment
- *     0.9"); the formula used is the usual one of the paper's platform:
+ *     only named as hyper-parameters in Section IV-A (their values, no formula);
+ *     the formula used is the usual one of the paper's platform:
  *     g' = g + lambda*w;  m <- mu*m + g' (m_0 = 0);  w <- w - eta*m.
  *   - Snapshot: the bracketed term of Eq. 2, second branch: each worker's weights
  *     right after the local step that closes a tau-block (Fig. 2 narrative:
- *     "after 3 local updates" for tau = 3).
+ *     with tau = 3 the averaging starts once three local updates are done).
  *   - Worker-axis mean: the (1/M) * sum_j of Eq. 2 (right-multiplication by J in
  *     the matrix form of Appendix "Matrix Representation").
  *   - Delayed merge: Eq. 2, second branch, appendix condition (k+1-d) mod tau = 0:

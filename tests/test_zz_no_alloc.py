@@ -5,7 +5,8 @@ is frozen once warm, as a plug-in that is handed a fixed arena, or beside anothe
 the device allocator.  For them the library
 carries its own 4 MiB mean vector.  The test drives the new call through the C ABI twice in a row (the
 built-in vector keeps the first call's contents, which must not leak into the second) and checks each
-result against the ordinary snapshot / average / merge entry points, which use caller-provided buffers.
+result against the ordinary snapshot / average / merge entry points, which use caller-provided buffers, and
+against the CPU oracle run with a delay of 0 (snapshot, mean and blend in one go).
 This file sorts last on purpose: a run that stops at the first failure has then run every other test.
 """
 import ctypes
@@ -28,10 +29,11 @@ def test_noalloc_rejects_sizes_beyond_its_built_in_vector():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("K,P,ld", [(8, 300_001, 300_008), (3, 1_048_576, 1_048_576), (5, 7, 7)])
-def test_noalloc_matches_the_buffered_entry_points_twice_in_a_row(K, P, ld):
+@pytest.mark.parametrize("K,P,ld,xi", [(8, 300_001, 300_008, 0.25), (3, 1_048_576, 1_048_576, 0.25), (5, 7, 7, 0.25),
+                                       (1, 4099, 4104, 0.5), (4, 70_000, 70_000, 0.0), (4, 70_000, 70_000, 1.0)])
+def test_noalloc_matches_the_buffered_entry_points_twice_in_a_row(K, P, ld, xi):
+    from oracle import OracleDaSGD
     from paper_2006_00441_b200 import binding as B
-    xi = 0.25
     gen = torch.Generator(device="cpu").manual_seed(K * 1000 + P % 997)
     stream = torch.cuda.Stream()
     for call in range(2):
@@ -53,5 +55,9 @@ def test_noalloc_matches_the_buffered_entry_points_twice_in_a_row(K, P, ld):
         assert_close(got, want, TOL_STEP, f"call {call}")
         exact = xi * W.double() + (1 - xi) * W.double().mean(0, keepdim=True)
         assert_close(got, exact.numpy(), TOL_STEP, f"call {call} vs definition")
+        cpu = OracleDaSGD(K, P, 1, 0, xi)
+        cpu.set_state(W.numpy())
+        cpu.snapshot(); cpu.average(); cpu.merge()
+        assert_close(got, cpu.w, TOL_STEP, f"call {call} vs the oracle")
         if ld > P:
             assert float(w[:, P:].abs().max()) == 0.0
