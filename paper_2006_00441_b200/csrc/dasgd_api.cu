@@ -1083,13 +1083,18 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
   const int G = C >= 16 ? C / 8 : 1;
   auto group_end = [&](int i) { const int e = (i / G + 1) * G - 1; return e < C - 1 ? e : C - 1; };
   std::vector<int> waited(n_lanes, -1);
-  for (int i = 0; i < C; ++i) {
+  // An iteration that only merges (no snapshot follows it) has no mean to feed, so the ranges of a group go
+  // out as one launch: the group is the granularity of the waits anyway.
+  const int stride = s_due ? 1 : G;
+  for (int i = 0; i < C; i += stride) {
+    const int last = i + stride - 1 < C - 1 ? i + stride - 1 : C - 1;   // last range of this launch
     const long long col0 = (long long)i * c->chunk_cols;
-    const long long len = c->cfg.P - col0 < c->chunk_cols ? c->cfg.P - col0 : c->chunk_cols;
-    const int li = i % n_lanes;
+    const long long col1 = (long long)(last + 1) * c->chunk_cols < c->cfg.P ? (long long)(last + 1) * c->chunk_cols : c->cfg.P;
+    const long long len = col1 - col0;
+    const int li = (i / stride) % n_lanes;
     cudaStream_t lane = li ? c->lanes[li - 1] : c->s0;
-    if (per_chunk_wait && waited[li] < group_end(i)) {
-      const int e = group_end(i);
+    if (per_chunk_wait && waited[li] < group_end(last)) {
+      const int e = group_end(last);
       stall_about_to_wait(c, c->slots[ms].stall_sp_c[e], lane);
       CU(c, cudaStreamWaitEvent(lane, c->slots[ms].e_avg_c[e], 0));
       waited[li] = e;
