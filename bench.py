@@ -455,6 +455,26 @@ def measure_workload(bench, wl, sched, steps, warmup, repeats, ring, lr, with_al
     return out
 
 
+def calibrate_chunks(bench, wl, sched, ring, lr):
+    """The number of column ranges is a trade between L2 residency (more, smaller ranges) and the host's
+    enqueue rate (four CUDA calls per range; a slower host needs fewer, longer ranges).  The formula in
+    auto_chunks assumes a host like the one it was tuned on, so a short trial decides: 40 steps at each of a few
+    counts around the formula's value, the fastest wins.  Returns the schedule with the chosen count."""
+    base = sched["n_chunks"]
+    cands = sorted({max(2, int(round(base * f))) for f in (0.6, 0.8, 1.0, 1.25)})
+    RING = len(ring)
+    trials = {}
+    for c in cands:
+        trial = dict(sched, n_chunks=c)
+        eng = bench.make(wl, trial)
+        r = bench.repeated(eng, 40, 5, 1, lambda e, t: e.step(ring[t % RING], lr))
+        trials[c] = r["ms_per_step"]
+        eng.close()
+        del eng
+    best = min(trials, key=trials.get)
+    return dict(sched, n_chunks=best, calibration_ms_per_step={str(k): round(v, 5) for k, v in trials.items()})
+
+
 def hidden_cost(wl, sched, ms_per_step, alone):
     """1 - (cycle time - cycle time of the main-stream kernels alone) / mean kernel alone."""
     if not all(k in alone for k in ("local_step", "mean", "merge")):
@@ -483,6 +503,8 @@ def run_ours(args, wl, name, bench=None, compact=False):
     def dev_step(e, t):
         e.step(ring[t % RING], lr)
 
+    if sched["merge"] == "chunked" and args.chunks == 0 and bench.comm is None and not args.no_calibrate:
+        sched = calibrate_chunks(bench, wl, sched, ring, lr)
     sampler = ClockSampler(bench.local_rank) if rank == 0 and not compact else None
     m = measure_workload(bench, wl, sched, args.steps, args.warmup, args.repeats, ring, lr,
                          with_alone=(not compact) or args.sweep)
@@ -783,6 +805,8 @@ def main():
     ap.add_argument("--shard", default="replicas", choices=["replicas", "workers"],
                     help="replicas: every GPU runs its own copy of the workload (default).  workers: the K workers of "
                          "every GPU are shards of one K*N-worker job; the partial sums are all-reduced over NCCL")
+    ap.add_argument("--no-calibrate", action="store_true",
+                    help="take the number of column ranges from the formula without the short trial")
     ap.add_argument("--sweep", action="store_true", help="run the K x tau x d sweep instead (one JSON line per point)")
     args = ap.parse_args()
     if args.warmup < 3:

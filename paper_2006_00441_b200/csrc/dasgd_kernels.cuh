@@ -128,8 +128,10 @@ __device__ __forceinline__ float blend_delta(float w, float mean, float snap) {
 // every CTA wave on one contiguous address range (measured 1.2 % faster).
 // MERGE: 0 none, 1 xi-blend, 2 delta.  SNAP: also store the final w into snap_out.
 
+// Three CTAs per SM (at most 80 registers): with a merge folded in the kernel would otherwise take 85-96
+// registers and lose a third of its resident warps, i.e. of its loads in flight.
 template <bool BF16, bool MOM, int MERGE, bool SNAP>
-__global__ void __launch_bounds__(kThreads) k_local_step_vec(const Params p) {
+__global__ void __launch_bounds__(kThreads, 3) k_local_step_vec(const Params p) {
   constexpr int EPU = BF16 ? 8 : 4;   // elements per unit
   constexpr int F4 = EPU / 4;          // float4 per unit
   constexpr int UNROLL = BF16 ? 2 : 4; // units per thread
