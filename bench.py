@@ -47,7 +47,7 @@ WORKLOADS = {
 }
 METRIC = "replica-param updates/s"
 UNIT = "updates/s"
-CHUNK_BYTES = 18 << 20   # target size of one column range of the weight array in the d = 1 pipeline
+CHUNK_BYTES = 18 << 20   # target size of one column range of the weight array in the column-range pipeline
 HOST_US_PER_RANGE = 20.0  # host time to enqueue one range (four CUDA calls, about 14 us measured) with some margin:
                           # more ranges than the iteration has time for would make the host the bottleneck
 MIN_RANGE_COLS = 409_600  # narrower ranges leave the mean kernel too few columns to fill the GPU (K >= 16)
@@ -61,7 +61,7 @@ def step_bytes(wl):
 
 
 def auto_chunks(K, P, bytes_per_update=25.0):
-    """Column ranges of the d = 1 pipeline: ranges of about CHUNK_BYTES of the [K][P] weight array (small enough
+    """Column ranges of the pipeline: ranges of about CHUNK_BYTES of the [K][P] weight array (small enough
     that the mean of a range finds much of it still in L2), but no more than the host can enqueue in the time
     the GPU needs for one iteration (estimated at the measured copy bandwidth)."""
     by_size = round(K * P * 4 / CHUNK_BYTES)
@@ -73,11 +73,11 @@ def schedule_of(wl, args):
     """How bench.py runs dasgd_step for this workload: {'merge': 'chunked'|'fused'|'separate', 'n_chunks', 'lanes'}."""
     if args.no_fuse:
         return {"merge": "separate", "n_chunks": 0, "lanes": 0, "copy_snapshot": True}
-    if wl["d"] >= 2:
-        return {"merge": "fused", "n_chunks": 0, "lanes": 0}
-    if wl["d"] == 1 and args.chunks != 1 and wl["P"] >= 2 * 4096:
+    if wl["d"] >= 1 and args.chunks != 1 and wl["P"] >= 2 * 4096:
         n = args.chunks if args.chunks > 0 else auto_chunks(wl["K"], wl["P"])
         return {"merge": "chunked", "n_chunks": n, "lanes": 1 if args.lanes else 0, "graph": 1 if args.graph else 0}
+    if wl["d"] >= 2:
+        return {"merge": "fused", "n_chunks": 0, "lanes": 0}
     return {"merge": "separate", "n_chunks": 0, "lanes": 0}
 
 
@@ -800,7 +800,7 @@ def main():
     ap.add_argument("--lanes", type=int, default=1, help="1: alternate the column ranges between two streams; 0: one stream")
     ap.add_argument("--graph", type=int, default=0, help="1: replay each chunked iteration from a CUDA graph")
     ap.add_argument("--chunks", type=int, default=0,
-                    help="column ranges of the d = 1 pipeline (merge folded into the step kernel); 0: by size "
+                    help="column ranges of the pipeline (merge folded into the step kernel); 0: by size "
                          "(ranges of about 18 MiB of weights); 1: off (separate merge kernel)")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "workers"],
                     help="replicas: every GPU runs its own copy of the workload (default).  workers: the K workers of "

@@ -131,12 +131,13 @@ typedef struct dasgd_config {
   int32_t n_stage;      /* gradient staging arrays behind g_stage: 0 (none), 1, or 2 (the copy of the
                            next step's gradients then overlaps this step's kernels)                   */
   int32_t n_chunks;     /* 0 or 1: off.  C > 1 (at most 1024; needs d >= 1, DASGD_FLAG_ROTATE_SNAPSHOT and
-                           DASGD_FLAG_FUSE_MERGE): when d == 1, dasgd_step cuts the parameter axis into C
-                           column ranges and pipelines them: the step kernel of range c (which blends the
-                           mean of range c that lands) is followed on the side stream by the mean of range
-                           c of the new snapshot, which runs beside the step kernels of ranges c+1, ...
-                           The merge then costs no pass of its own although the mean of step s is consumed
-                           by step s+1.  Results are the same as without chunks.                        */
+                           DASGD_FLAG_FUSE_MERGE): dasgd_step cuts the parameter axis into C column ranges
+                           and pipelines them: the step kernel of range c (which blends the mean of range c
+                           that lands) is followed on the side stream by the mean of range c of the new
+                           snapshot, which runs beside the step kernels of ranges c+1, ...  With d == 1 the
+                           merge then costs no pass of its own although the mean of step s is consumed by
+                           step s+1; with any d >= 1 the mean of a range starts while much of the range is
+                           still in the L2 cache.  Results are the same as without chunks.               */
   void *w;              /* device, [K][ld] float32, in/out: weights (master weights in bf16 mode); with
                            DASGD_FLAG_ROTATE_SNAPSHOT: where the weights START (see dasgd_get_weights)  */
   void *m;              /* device, [K][ld] float32, in/out: momentum buffers (start them at 0)        */

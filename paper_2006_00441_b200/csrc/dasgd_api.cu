@@ -694,7 +694,7 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
   for (int i = 0; c.snap && i < c.n_slots; ++i)
     ctx->pool.push_back(static_cast<float *>(c.snap) + (size_t)i * c.K * c.ld);
   ctx->frozen.assign(ctx->pool.size(), 0);
-  if (c.n_chunks > 1 && c.d == 1) {  // only d == 1 needs the pipeline: for d >= 2 the mean has a whole step
+  if (c.n_chunks > 1 && c.d >= 1) {
     const long long tile = 4096;     // columns per CTA of the vector step kernels, both dtypes
     const long long tiles = (c.P + tile - 1) / tile;
     const long long per = (tiles + c.n_chunks - 1) / c.n_chunks;
@@ -909,13 +909,15 @@ dasgd_status step_inline(dasgd_ctx *c, const void *grads, float lr, bool m_due, 
   return DASGD_OK;
 }
 
-// One iteration of the chunked pipeline (d == 1, rotating snapshots, merge folded into the step kernel).
+// One iteration of the chunked pipeline (d >= 1, rotating snapshots, merge folded into the step kernel).
 // Per column range i, on the main stream: wait for range i of the mean that lands (computed one
 // iteration ago, so normally long finished), run the step kernel on range i; if a snapshot is due,
 // record "range i written" and let the side stream average range i of the new weights while the main
-// stream goes on with ranges i+1, ...  The mean of range i thus has the rest of this iteration and the
-// first i ranges of the next one as its window (the condition t_c < d*t_p of Eq. 6, per range), although
-// the next iteration's kernels consume it directly.
+// stream goes on with ranges i+1, ...  With d == 1 the mean of range i thus has the rest of this iteration
+// and the first i ranges of the next one as its window (the condition t_c < d*t_p of Eq. 6, per range),
+// although the next iteration's kernels consume it directly.  With d >= 2 the window is there anyway; what
+// the pipeline still buys is that the mean of a range reads weights that were written a moment ago and
+// are largely still in L2.
 // The launches of one chunked iteration, enqueued on the main stream, the extra lanes and the side stream.
 // Used while a stream capture is active; `ev` are capture-only events.
 dasgd_status enqueue_chunked(dasgd_ctx *c, const Params &p, const Params &q, int mode, bool vec, bool s_due) {

@@ -21,7 +21,7 @@ FUSED = 0x4 | 0x8 | 0x100   # snapshots by array rotation; merge folded into the
 def chunks_for(K, P, d):
     """The benchmark's policy for the number of column ranges."""
     import bench
-    return bench.auto_chunks(K, P) if d == 1 and P >= 2 * 4096 else 0
+    return bench.auto_chunks(K, P) if d >= 1 and P >= 2 * 4096 else 0
 
 
 @pytest.fixture(scope="module")
