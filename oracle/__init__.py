@@ -59,6 +59,8 @@ def bind(path: str) -> ctypes.CDLL:
     L.oracle_dasgd_merge.argtypes = [vp]
     L.oracle_dasgd_step.argtypes = [vp, vp, f32]
     L.oracle_dasgd_set_variant.argtypes = [vp, i32, i32]
+    L.oracle_dasgd_set_momentum_averaging.argtypes = [vp, i32]
+    L.oracle_dasgd_get_pending_momentum.argtypes = [vp, i32, vp, vp]
     L.oracle_dasgd_set_shard.argtypes = [vp, i32]
     L.oracle_dasgd_partial_sum.argtypes = [vp, vp]
     L.oracle_dasgd_set_mean_from_sum.argtypes = [vp, vp]
@@ -103,7 +105,7 @@ class OracleDaSGD:
     """K replicas of a P-vector driven by the oracle.  Arrays are numpy, [K][P]."""
 
     def __init__(self, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=F32,
-                 merge_mode=MERGE_XI, omp=False, nesterov=False, decoupled_wd=False):
+                 merge_mode=MERGE_XI, omp=False, nesterov=False, decoupled_wd=False, average_momentum=False):
         self._L = _lib(omp)
         self.K, self.P, self.tau, self.d, self.dtype = K, P, tau, d, dtype
         self._h = self._L.oracle_dasgd_create(K, P, tau, d, xi, momentum, weight_decay, dtype, merge_mode)
@@ -111,6 +113,8 @@ class OracleDaSGD:
             raise OracleError("invalid configuration")
         if (nesterov or decoupled_wd) and self._L.oracle_dasgd_set_variant(self._h, int(nesterov), int(decoupled_wd)) != 0:
             raise OracleError("invalid variant (Nesterov needs momentum)")
+        if average_momentum and self._L.oracle_dasgd_set_momentum_averaging(self._h, 1) != 0:
+            raise OracleError("momentum averaging needs momentum > 0")
 
     def close(self):
         if getattr(self, "_h", None):
@@ -177,6 +181,12 @@ class OracleDaSGD:
         self._chk(self._L.oracle_dasgd_get_pending(self._h, i, ctypes.byref(s), _ptr(snap), _ptr(mean)),
                   "get_pending")
         return s.value, snap, mean
+
+    def pending_momentum(self, i=0, want_mean=True):
+        snap = np.empty((self.K, self.P), np.float32)
+        mean = np.empty((self.P,), np.float32) if want_mean else None
+        self._chk(self._L.oracle_dasgd_get_pending_momentum(self._h, i, _ptr(snap), _ptr(mean)), "get_pending_momentum")
+        return snap, mean
 
     def local_step(self, g, lr):
         self._chk(self._L.oracle_dasgd_local_step(self._h, _ptr(self._grad(g)), lr), "local_step")

@@ -36,6 +36,8 @@ struct Pending {
   int64_t s;                // number of completed local steps when the snapshot was taken
   std::vector<float> snap;  // [K][P]
   std::vector<float> mean;  // [P]
+  std::vector<float> snap_m;  // [K][P] momentum buffers at the snapshot (momentum averaging only)
+  std::vector<float> mean_m;  // [P]
   bool averaged;
 };
 
@@ -47,6 +49,7 @@ struct oracle_dasgd {
   int64_t P;
   float xi, momentum, weight_decay;
   bool nesterov = false, decoupled_wd = false;
+  bool average_momentum = false;  // the momentum buffers go through snapshot, mean and merge like the weights
   int64_t t;  // completed local steps
   std::vector<float> w, m;
   std::vector<uint16_t> w_lp;
@@ -79,6 +82,12 @@ int oracle_dasgd_set_variant(oracle_dasgd *o, int32_t nesterov, int32_t decouple
   if (!o || (nesterov && o->momentum == 0.0f)) return ORACLE_ERR_ARG;
   o->nesterov = nesterov != 0;
   o->decoupled_wd = decoupled_wd != 0;
+  return ORACLE_OK;
+}
+
+int oracle_dasgd_set_momentum_averaging(oracle_dasgd *o, int32_t on) {
+  if (!o || (on && o->momentum == 0.0f) || !o->pending.empty()) return ORACLE_ERR_ARG;
+  o->average_momentum = on != 0;
   return ORACLE_OK;
 }
 
@@ -122,6 +131,17 @@ int oracle_dasgd_get_pending(const oracle_dasgd *o, int32_t i, int64_t *s, float
   return ORACLE_OK;
 }
 
+int oracle_dasgd_get_pending_momentum(const oracle_dasgd *o, int32_t i, float *snap_m, float *mean_m) {
+  if (!o || !o->average_momentum || i < 0 || i >= static_cast<int32_t>(o->pending.size())) return ORACLE_ERR_ARG;
+  const Pending &q = o->pending[i];
+  if (snap_m) std::memcpy(snap_m, q.snap_m.data(), q.snap_m.size() * sizeof(float));
+  if (mean_m) {
+    if (!q.averaged) return ORACLE_ERR_STATE;
+    std::memcpy(mean_m, q.mean_m.data(), q.mean_m.size() * sizeof(float));
+  }
+  return ORACLE_OK;
+}
+
 // Eq. 2, first branch, with the momentum / weight-decay form stated in the header.
 int oracle_dasgd_local_step(oracle_dasgd *o, const void *g, float lr) {
   if (!o || !g) return ORACLE_ERR_ARG;
@@ -157,6 +177,7 @@ int oracle_dasgd_snapshot(oracle_dasgd *o) {
   Pending q;
   q.s = o->t;
   q.snap = o->w;
+  if (o->average_momentum) q.snap_m = o->m;
   q.averaged = false;
   o->pending.push_back(std::move(q));
   return ORACLE_OK;
@@ -178,6 +199,15 @@ int oracle_dasgd_average(oracle_dasgd *o) {
     for (int32_t k = 0; k < o->K; ++k) acc += static_cast<double>(q->snap[static_cast<size_t>(k) * P + p]);
     q->mean[p] = static_cast<float>(acc / static_cast<double>(o->K));
   }
+  if (o->average_momentum) {  // the same (1/M) * sum over workers, applied to the momentum buffers
+    q->mean_m.assign(static_cast<size_t>(P), 0.0f);
+#pragma omp parallel for schedule(static)
+    for (int64_t p = 0; p < P; ++p) {
+      double acc = 0.0;
+      for (int32_t k = 0; k < o->K; ++k) acc += static_cast<double>(q->snap_m[static_cast<size_t>(k) * P + p]);
+      q->mean_m[p] = static_cast<float>(acc / static_cast<double>(o->K));
+    }
+  }
   q->averaged = true;
   return ORACLE_OK;
 }
@@ -187,7 +217,7 @@ int oracle_dasgd_average(oracle_dasgd *o) {
 // then a two-level sum: each holder adds up its own workers, the partial sums are added across
 // holders (by the caller), and the total is divided by M = K_total once.
 int oracle_dasgd_set_shard(oracle_dasgd *o, int32_t K_total) {
-  if (!o || K_total < o->K) return ORACLE_ERR_ARG;
+  if (!o || K_total < o->K || o->average_momentum) return ORACLE_ERR_ARG;
   o->K_total = K_total;
   return ORACLE_OK;
 }
@@ -241,6 +271,13 @@ int oracle_dasgd_merge(oracle_dasgd *o) {
       else
         o->w[i] = static_cast<float>(wi + (avg - static_cast<double>(q.snap[i])));
       if (bf16) o->w_lp[i] = f32_to_bf16_rne(o->w[i]);
+      if (o->average_momentum) {  // the same blend on the momentum buffer, with the stale mean of the buffers
+        const double mi = o->m[i], avg_m = q.mean_m[p];
+        if (o->merge_mode == ORACLE_MERGE_XI)
+          o->m[i] = static_cast<float>(xi * mi + one_minus_xi * avg_m);
+        else
+          o->m[i] = static_cast<float>(mi + (avg_m - static_cast<double>(q.snap_m[i])));
+      }
     }
   }
   o->pending.pop_front();

@@ -62,6 +62,17 @@ void oracle_dasgd_destroy(oracle_dasgd *o);
  *                  torch.optim.SGD without weight decay, and the closed form (1-eta*lambda)^T for zero gradients) */
 int oracle_dasgd_set_variant(oracle_dasgd *o, int32_t nesterov, int32_t decoupled_wd);
 
+/* Momentum averaging (NOT in the paper, which averages weights only): the momentum buffers go through the same
+ * three operations as the weights -- copied at the snapshot, averaged over the workers, and blended back d steps
+ * later with the same xi (or, in merge_mode 1, m <- m + (mean_m - snapshot_m)).  Needs momentum > 0; may only be
+ * switched while no snapshot is pending; not available on a shard of the worker axis.
+ * Pinned: identical workers stay identical and follow plain momentum SGD; xi = 1 changes nothing; with xi = 0 and
+ * d = 0 every buffer equals the mean of the buffers right after a merge; the worker-mean of the buffers is
+ * preserved by a d = 0 merge; a hand-worked trajectory (tests/golden). */
+int oracle_dasgd_set_momentum_averaging(oracle_dasgd *o, int32_t on);
+/* momentum snapshot [K][P] / its mean [P] of the i-th oldest pending snapshot; either may be NULL */
+int oracle_dasgd_get_pending_momentum(const oracle_dasgd *o, int32_t i, float *snap_m, float *mean_m);
+
 /* State access: w, m are [K][P] float32 (row k = worker k); w_lp is [K][P] bf16 bits. */
 int oracle_dasgd_set_state(oracle_dasgd *o, const float *w, const float *m);
 int oracle_dasgd_get_state(const oracle_dasgd *o, float *w, float *m, uint16_t *w_lp);

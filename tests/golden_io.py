@@ -14,7 +14,7 @@ def load(name):
             if not line:
                 continue
             key, rest = line[0], line[1:]
-            if key in ("K", "P", "tau", "d", "merge_mode"):
+            if key in ("K", "P", "tau", "d", "merge_mode", "average_momentum"):
                 cfg[key] = int(rest[0])
             elif key in ("xi", "lr", "momentum", "weight_decay"):
                 cfg[key] = float(rest[0])
@@ -26,6 +26,8 @@ def load(name):
                 exp_w[(int(rest[0]), int(rest[1]))] = [float(v) for v in rest[2:]]
             elif key == "expect_m":
                 exp_m[(int(rest[0]), int(rest[1]))] = [float(v) for v in rest[2:]]
+            elif key == "expect_mean_m":     # mean of the momentum buffers of the snapshot taken at that step
+                cfg.setdefault("expect_mean_m", {})[int(rest[0])] = [float(v) for v in rest[1:]]
             elif key == "expect_mean":
                 exp_mean[int(rest[0])] = [float(v) for v in rest[1:]]
             else:

@@ -6,15 +6,16 @@ from oracle import OracleDaSGD
 from tests.golden_io import load
 
 CASES = ["w1_xi_blend.txt", "w2_momentum.txt", "w3_d_equals_tau.txt", "w4_delta_merge.txt",
-         "w1_stacked_p8.txt"]
+         "w1_stacked_p8.txt", "w5_momentum_averaging.txt"]
 
 
 @pytest.mark.parametrize("name", CASES)
 def test_golden_trajectory(name):
     cfg, W0, G, exp_w, exp_m, exp_mean = load(name)
     o = OracleDaSGD(cfg["K"], cfg["P"], cfg["tau"], cfg["d"], cfg["xi"], cfg["momentum"],
-                    cfg["weight_decay"], merge_mode=cfg["merge_mode"])
+                    cfg["weight_decay"], merge_mode=cfg["merge_mode"], average_momentum=bool(cfg.get("average_momentum")))
     o.set_state(W0)
+    exp_mean_m = cfg.get("expect_mean_m", {})
     seen_w = seen_m = seen_mean = 0
     for t in range(G.shape[0]):
         o.step(G[t], cfg["lr"])
@@ -33,4 +34,8 @@ def test_golden_trajectory(name):
             assert s == u
             np.testing.assert_array_equal(mean, np.array(exp_mean[u], np.float32), err_msg=f"mean s={u}")
             seen_mean += 1
-    assert seen_w == len(exp_w) and seen_m == len(exp_m) and seen_mean == len(exp_mean)
+        if u in exp_mean_m:
+            _, mean_m = o.pending_momentum(o.n_pending - 1)
+            np.testing.assert_array_equal(mean_m, np.array(exp_mean_m[u], np.float32), err_msg=f"mean of m s={u}")
+            seen_mean += 1
+    assert seen_w == len(exp_w) and seen_m == len(exp_m) and seen_mean == len(exp_mean) + len(exp_mean_m)

@@ -383,3 +383,160 @@ def test_pending_queue_depth_and_explicit_calls_match_step(tau, d):
                 b.merge()
         np.testing.assert_array_equal(a.w, b.w)
         assert a.n_pending == b.n_pending <= max(1, -(-d // tau))
+
+
+# ---------------------------------------------------------------- momentum averaging (a variant, not in the paper)
+
+def _independent_period(w, m, G, lr, mu):
+    """tau plain momentum-SGD steps of every worker from the state (w, m): a run with xi = 1 (no merge acts)."""
+    K, P = w.shape
+    o = OracleDaSGD(K, P, tau=G.shape[0] + 1, d=1, xi=1.0, momentum=mu)
+    o.set_state(w, m)
+    for t in range(G.shape[0]):
+        o.step(G[t], lr)
+    return o.w.astype(np.float64), o.m.astype(np.float64)
+
+
+@pytest.mark.parametrize("xi", [0.0, 0.25, 1.0])
+def test_momentum_averaging_without_delay_blends_both_halves_of_the_state(xi):
+    """d = 0: right after a merge, w_k = xi*w_k' + (1-xi)*mean(w') and m_k = xi*m_k' + (1-xi)*mean(m'), where the
+    primed state is what tau independent momentum-SGD steps give (taken from runs in which no merge acts).
+    xi = 0: every worker then holds the same weights and the same buffer; any xi: the worker-mean of the buffers
+    is untouched by the merge."""
+    K, P, tau, lr, mu = 3, 19, 3, 0.1, 0.8
+    G = rng_grads(3 * tau, K, P, 40)
+    w = np.random.default_rng(41).standard_normal((K, P)).astype(np.float32)
+    m = np.zeros((K, P), np.float32)
+    o = OracleDaSGD(K, P, tau=tau, d=0, xi=xi, momentum=mu, average_momentum=True)
+    o.set_state(w)
+    for period in range(3):
+        Gp = G[period * tau:(period + 1) * tau]
+        for t in range(tau):
+            o.step(Gp[t], lr)
+        wp, mp = _independent_period(w, m, Gp, lr, mu)
+        xi64 = np.float64(np.float32(xi))
+        w_want = xi64 * wp + (1 - xi64) * wp.mean(axis=0)
+        m_want = xi64 * mp + (1 - xi64) * mp.mean(axis=0)
+        np.testing.assert_allclose(o.w, w_want, rtol=0, atol=2e-6)
+        np.testing.assert_allclose(o.m, m_want, rtol=0, atol=2e-6)
+        np.testing.assert_allclose(o.m.astype(np.float64).mean(axis=0), mp.mean(axis=0), rtol=0, atol=2e-6)
+        if xi == 0.0:
+            assert np.ptp(o.w, axis=0).max() == 0.0 and np.ptp(o.m, axis=0).max() == 0.0
+        w, m = o.w, o.m
+
+
+@pytest.mark.parametrize("tau,d", [(1, 1), (2, 1), (3, 2), (2, 2), (1, 2)])
+def test_momentum_averaging_is_a_no_op_at_xi_one(tau, d):
+    K, P, T = 3, 23, 12
+    G = rng_grads(T, K, P, 42)
+    w0 = np.random.default_rng(43).standard_normal((K, P)).astype(np.float32)
+    a = OracleDaSGD(K, P, tau, d, xi=1.0, momentum=0.9, weight_decay=0.01, average_momentum=True)
+    b = OracleDaSGD(K, P, tau, d, xi=1.0, momentum=0.9, weight_decay=0.01)
+    a.set_state(w0); b.set_state(w0)
+    for t in range(T):
+        a.step(G[t], 0.1); b.step(G[t], 0.1)
+    np.testing.assert_array_equal(a.w, b.w)
+    np.testing.assert_array_equal(a.m, b.m)
+
+
+@pytest.mark.parametrize("tau,d,xi", [(2, 1, 0.25), (3, 2, 0.5), (2, 2, 0.0), (1, 2, 0.25)])
+def test_momentum_averaging_uses_the_stale_mean_of_the_buffers(tau, d, xi):
+    """Zero gradients, no decay: a buffer only decays, m(t) = mu^t m(0), so the first merge (at step tau+d, of the
+    snapshot taken at step tau) must give m_k = xi*mu^(tau+d)*m_k(0) + (1-xi)*mu^tau*mean(m(0)): the mean is the
+    one of d steps ago, not the current one."""
+    K, P, mu = 4, 9, 0.5
+    r = np.random.default_rng(44)
+    m0 = r.standard_normal((K, P)).astype(np.float32)
+    o = OracleDaSGD(K, P, tau, d, xi=xi, momentum=mu, average_momentum=True)
+    o.set_state(r.standard_normal((K, P)).astype(np.float32), m0)
+    Z = np.zeros((K, P), np.float32)
+    for t in range(tau + d):                   # no merge lands before step tau + d
+        np.testing.assert_allclose(o.m, mu ** t * m0.astype(np.float64), rtol=0, atol=1e-6)
+        o.step(Z, 0.1)
+    xi64 = np.float64(np.float32(xi))
+    want = xi64 * mu ** (tau + d) * m0.astype(np.float64) + (1 - xi64) * mu ** tau * m0.astype(np.float64).mean(axis=0)
+    np.testing.assert_allclose(o.m, want, rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("tau,d", [(2, 1), (1, 1), (3, 2), (1, 2)])
+def test_momentum_averaging_delta_form_keeps_the_mean_buffer_on_its_plain_recursion(tau, d):
+    """merge_mode 1: m_k <- m_k + (mean(m^) - m^_k) adds corrections that sum to zero over the workers, so the
+    worker-mean of the buffers obeys mean_m <- mu*mean_m + mean(g) at every step, merges or not."""
+    K, P, T, mu = 4, 13, 14, 0.7
+    G = rng_grads(T, K, P, 45)
+    o = OracleDaSGD(K, P, tau, d, xi=0.25, momentum=mu, merge_mode=MERGE_DELTA, average_momentum=True)
+    o.set_state(np.random.default_rng(46).standard_normal((K, P)).astype(np.float32))
+    mean_m = np.zeros(P)
+    moved = False
+    plain = OracleDaSGD(K, P, tau, d, xi=0.25, momentum=mu, merge_mode=MERGE_DELTA)
+    plain.set_state(o.w)
+    for t in range(T):
+        o.step(G[t], 0.05); plain.step(G[t], 0.05)
+        mean_m = np.float64(np.float32(mu)) * mean_m + G[t].astype(np.float64).mean(axis=0)
+        np.testing.assert_allclose(o.m.astype(np.float64).mean(axis=0), mean_m, rtol=0, atol=5e-6)
+        moved = moved or np.abs(o.m - plain.m).max() > 1e-3
+    assert moved      # the buffers themselves do differ from the run without momentum averaging
+
+
+def test_momentum_averaging_identical_workers():
+    """Identical workers with identical gradients stay identical; with d = 0 the merge is then the identity and the
+    run is plain momentum SGD (torch.optim.SGD)."""
+    K, P, T, lr, mu = 3, 11, 10, 0.1, 0.9
+    g1 = rng_grads(T, 1, P, 47)
+    G = np.repeat(g1, K, axis=1)
+    w0 = np.random.default_rng(48).standard_normal(P).astype(np.float32)
+    for tau, d in [(2, 1), (1, 2), (2, 0)]:
+        o = OracleDaSGD(K, P, tau, d, xi=0.25, momentum=mu, average_momentum=True)
+        o.set_state(w0)
+        p = torch.tensor(w0, dtype=torch.float64, requires_grad=True)
+        opt = torch.optim.SGD([p], lr=float(np.float32(lr)), momentum=float(np.float32(mu)))
+        for t in range(T):
+            o.step(G[t], lr)
+            p.grad = torch.tensor(g1[t, 0], dtype=torch.float64)
+            opt.step()
+            assert np.ptp(o.w, axis=0).max() == 0.0 and np.ptp(o.m, axis=0).max() == 0.0
+            if d == 0:
+                np.testing.assert_allclose(o.w[0], p.detach().numpy(), rtol=2e-6, atol=2e-6)
+
+
+def test_momentum_averaging_needs_momentum_and_an_unsharded_worker_axis():
+    from oracle import OracleError
+    with pytest.raises(OracleError):
+        OracleDaSGD(2, 4, 1, 1, 0.5, momentum=0.0, average_momentum=True)
+    o = OracleDaSGD(2, 4, 1, 1, 0.5, momentum=0.9, average_momentum=True)
+    with pytest.raises(OracleError):
+        o.set_shard(4)
+
+
+def test_momentum_averaging_delta_form_without_delay_equalises_the_buffers():
+    """merge_mode 1 with d = 0: the snapshot is the current state, so m_k + (mean(m) - m_k) = mean(m) for every
+    worker (and likewise for the weights): the sign of the correction matters here."""
+    K, P, tau = 3, 7, 2
+    G = rng_grads(6, K, P, 49)
+    o = OracleDaSGD(K, P, tau, 0, xi=0.25, momentum=0.6, merge_mode=MERGE_DELTA, average_momentum=True)
+    o.set_state(np.random.default_rng(50).standard_normal((K, P)).astype(np.float32))
+    for t in range(6):
+        before_m = o.m.astype(np.float64)
+        o.step(G[t], 0.1)
+        if (t + 1) % tau == 0:
+            stepped = np.float64(np.float32(0.6)) * before_m + G[t]
+            np.testing.assert_allclose(o.m, np.broadcast_to(stepped.mean(axis=0), (K, P)), rtol=0, atol=2e-6)
+            np.testing.assert_allclose(np.ptp(o.w.astype(np.float64), axis=0), 0, atol=1e-6)
+
+
+def test_momentum_averaging_mean_is_that_of_the_snapshot_not_of_later_buffers():
+    """Explicit calls with a local step between the snapshot and its averaging: the mean must be the one of the
+    buffers as they were at the snapshot."""
+    K, P = 3, 5
+    G = rng_grads(3, K, P, 51)
+    o = OracleDaSGD(K, P, 4, 2, xi=0.5, momentum=0.9, average_momentum=True)
+    o.set_state(np.zeros(P, np.float32))
+    o.local_step(G[0], 0.1)
+    o.snapshot()
+    m_at_snapshot = o.m.astype(np.float64)
+    o.local_step(G[1], 0.1)
+    o.average()
+    snap_m, mean_m = o.pending_momentum(0)
+    np.testing.assert_array_equal(snap_m, m_at_snapshot.astype(np.float32))
+    np.testing.assert_allclose(mean_m, m_at_snapshot.mean(axis=0), rtol=0, atol=1e-6)
+    assert np.abs(o.m.astype(np.float64).mean(axis=0) - mean_m).max() > 1e-3

@@ -47,6 +47,13 @@ MUTATIONS = {
     "partial sum takes the newest snapshot": (
         "  const Pending *q = nullptr;\n  for (const auto &cand : o->pending)\n    if (!cand.averaged) { q = &cand; break; }",
         "  const Pending *q = nullptr;\n  for (const auto &cand : o->pending)\n    if (!cand.averaged) { q = &cand; }"),
+    "momentum averaging: blend takes the mean of the weights": ("avg_m = q.mean_m[p]", "avg_m = q.mean[p]"),
+    "momentum averaging: snapshot taken from the weights": ("q.snap_m = o->m;", "q.snap_m = o->w;"),
+    "momentum averaging: blend weights swapped": ("xi * mi + one_minus_xi * avg_m", "one_minus_xi * mi + xi * avg_m"),
+    "momentum averaging: delta sign": ("mi + (avg_m - static_cast<double>(q.snap_m[i]))", "mi - (avg_m - static_cast<double>(q.snap_m[i]))"),
+    "momentum averaging: fresh buffers instead of the snapshot": ("acc += static_cast<double>(q->snap_m[static_cast<size_t>(k) * P + p]);",
+                                                                  "acc += static_cast<double>(o->m[static_cast<size_t>(k) * P + p]);"),
+    "momentum averaging: switched on for everyone": ("bool average_momentum = false;", "bool average_momentum = true;"),
     "momentum merged too": ("o->pending.pop_front();\n  return ORACLE_OK;", "for (auto &x : o->m) x *= o->xi;\n  o->pending.pop_front();\n  return ORACLE_OK;"),
 }
 
@@ -74,6 +81,15 @@ def battery():
     I.test_decoupled_weight_decay_closed_form_with_momentum()
     I.test_bf16_rounding_matches_torch_cast()
     I.test_bf16_mode_master_equals_f32_run_on_widened_gradients()
+    for xi in (0.0, 0.25):
+        I.test_momentum_averaging_without_delay_blends_both_halves_of_the_state(xi)
+    I.test_momentum_averaging_is_a_no_op_at_xi_one(2, 1)
+    for args in [(2, 1, 0.25), (1, 2, 0.25)]:
+        I.test_momentum_averaging_uses_the_stale_mean_of_the_buffers(*args)
+    I.test_momentum_averaging_delta_form_keeps_the_mean_buffer_on_its_plain_recursion(2, 1)
+    I.test_momentum_averaging_identical_workers()
+    I.test_momentum_averaging_delta_form_without_delay_equalises_the_buffers()
+    I.test_momentum_averaging_mean_is_that_of_the_snapshot_not_of_later_buffers()
     S.test_mean_divides_by_the_total_number_of_workers()
     S.test_shards_in_one_process_reproduce_the_unsharded_oracle(2, 1, (3, 5))
     S.test_one_shard_holding_every_worker_is_the_unsharded_oracle_bit_for_bit()
