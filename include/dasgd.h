@@ -259,6 +259,23 @@ dasgd_status dasgd_get_kernel_units(dasgd_ctx *ctx, int32_t which, int64_t *unit
  * no rounding of the method's state happens outside the library.  DASGD_ERR_BAD_STATE in float32 mode. */
 dasgd_status dasgd_refresh_lp(dasgd_ctx *ctx);
 
+/* ---- Momentum averaging (a variant; the paper has no counterpart: Section III averages the weights only and
+ * Section IV-A says nothing about the momentum buffers at a merge, so by default they stay local).
+ *
+ * After this call the momentum buffers go through the same three operations as the weights, at the same moments:
+ * every snapshot also copies m into the slot's [K][ld] array of m_snap (main stream), every mean is followed by the
+ * worker-axis mean of that copy into the slot's [ld] vector of m_mean (side stream), and every merge also blends
+ * the buffers, m_k <- xi*m_k + (1-xi)*mean_m (DASGD_MERGE_DELTA: m_k <- m_k + (mean_m - copy_k)), after the kernels
+ * of that step have updated them.  These are passes of their own (8 + 4 + 4/K + 8 + 4/K bytes per
+ * replica-parameter and cycle, 4 more for the delta form): the variant is for studying the method, not for speed.
+ * m_snap: device, [n_slots][K][ld] float32; m_mean: device, [n_slots][ld] float32; both caller-owned, 16-byte
+ * aligned, on cfg.device, borrowed until dasgd_destroy.  Call it right after dasgd_init (DASGD_ERR_BAD_STATE once
+ * the context has been used).  Needs momentum > 0.  DASGD_ERR_UNSUPPORTED with DASGD_FLAG_INLINE_MEAN and on a
+ * sharded worker axis; DASGD_FLAG_GRAPH is ignored.  dasgd_get_pending_momentum: the copy and the mean of the i-th
+ * oldest pending snapshot (either pointer may be NULL). */
+dasgd_status dasgd_set_momentum_averaging(dasgd_ctx *ctx, void *m_snap_device, void *m_mean_device);
+dasgd_status dasgd_get_pending_momentum(const dasgd_ctx *ctx, int32_t i, void **m_snap_device, void **m_mean_device);
+
 /* ---- Sharded worker axis (the data-parallel setting of Section II-B: the M workers live on several GPUs
  * and an all-reduce adds their contributions; Section III: the averaging runs while the local steps go on).
  *

@@ -36,6 +36,7 @@ EXPORTS = [
     "dasgd_get_kernel_timing", "dasgd_reset_timing", "dasgd_get_launches", "dasgd_strerror", "dasgd_last_error", "dasgd_destroy", "dasgd_version",
     "dasgd_average_merge_noalloc", "dasgd_delay_guideline", "dasgd_advise_delay", "dasgd_export_state", "dasgd_import_state",
     "dasgd_get_kernel_units", "dasgd_refresh_lp",
+    "dasgd_set_momentum_averaging", "dasgd_get_pending_momentum",
     "dasgd_set_shard", "dasgd_set_shard_nccl", "dasgd_nccl_unique_id", "dasgd_nccl_comm_init", "dasgd_nccl_comm_destroy",
 ]
 
@@ -97,6 +98,8 @@ def _load() -> ctypes.CDLL:
     L.dasgd_advise_delay.argtypes = [vp, f64, pi32, pi32, pf64, pf64]
     L.dasgd_export_state.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
     L.dasgd_import_state.argtypes = [vp, vp, i64]
+    L.dasgd_set_momentum_averaging.argtypes = [vp, vp, vp]
+    L.dasgd_get_pending_momentum.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     L.dasgd_set_shard.argtypes = [vp, i32, EXCHANGE_FN, vp]
     L.dasgd_set_shard_nccl.argtypes = [vp, i32, vp]
     L.dasgd_nccl_unique_id.argtypes = [vp]
@@ -227,6 +230,16 @@ def dasgd_import_state(ctx, blob: bytes):
     _check(_L.dasgd_import_state(ctx, blob, len(blob)), ctx)
 
 
+def dasgd_set_momentum_averaging(ctx, m_snap_ptr: int, m_mean_ptr: int):
+    _check(_L.dasgd_set_momentum_averaging(ctx, m_snap_ptr, m_mean_ptr), ctx)
+
+
+def dasgd_get_pending_momentum(ctx, i: int):
+    snap, mean = ctypes.c_void_p(), ctypes.c_void_p()
+    _check(_L.dasgd_get_pending_momentum(ctx, i, ctypes.byref(snap), ctypes.byref(mean)), ctx)
+    return snap.value, mean.value
+
+
 def dasgd_set_shard(ctx, K_total: int, exchange, user=None):
     """`exchange`: an EXCHANGE_FN instance; the caller keeps it alive as long as the context."""
     _check(_L.dasgd_set_shard(ctx, K_total, exchange, user), ctx)
@@ -290,7 +303,7 @@ class DaSGD:
 
     def __init__(self, K, P, tau, d, xi, momentum=0.0, weight_decay=0.0, dtype=DASGD_F32,
                  merge_mode=DASGD_MERGE_XI, flags=0, n_slots=None, ld=None, device=0, host_staging=False,
-                 sync_timeout_ms=0, order_after_current=True, snapshot_arrays=True, n_chunks=0):
+                 sync_timeout_ms=0, order_after_current=True, snapshot_arrays=True, n_chunks=0, average_momentum=False):
         if not torch.cuda.is_available():
             raise RuntimeError("DaSGD needs a CUDA device; there is no CPU implementation")
         self.K, self.P, self.tau, self.d = K, P, tau, d
@@ -335,6 +348,15 @@ class DaSGD:
         self._host_refs = []
         torch.cuda.synchronize(dev)  # the zero fills above ran on torch's current stream
         self.ctx = dasgd_init(cfg)
+        self.m_snap = self.m_mean = None
+        if average_momentum:   # the variant in which the momentum buffers are averaged like the weights
+            self.m_snap = torch.empty((self.n_slots, K, self.ld), dtype=torch.float32, device=dev)
+            self.m_mean = torch.empty((self.n_slots, self.ld), dtype=torch.float32, device=dev)
+            try:
+                dasgd_set_momentum_averaging(self.ctx, self.m_snap.data_ptr(), self.m_mean.data_ptr())
+            except DasgdError:
+                self.close()
+                raise
 
     # -- state ---------------------------------------------------------------
     @property
@@ -412,6 +434,12 @@ class DaSGD:
         _, _, mean_ptr = dasgd_get_pending(self.ctx, i)
         slot = (mean_ptr - self.mean.data_ptr()) // (self.ld * 4)
         return self.mean[slot, :self.P]
+
+    def pending_momentum_mean(self, i=0) -> torch.Tensor:
+        """The mean of the momentum buffers of the i-th oldest pending snapshot (momentum averaging only)."""
+        _, mean_ptr = dasgd_get_pending_momentum(self.ctx, i)
+        slot = (mean_ptr - self.m_mean.data_ptr()) // (self.ld * 4)
+        return self.m_mean[slot, :self.P]
 
     def timing(self):
         """(averages completed, ms spent averaging on the side stream, ms the main stream waited for them)."""

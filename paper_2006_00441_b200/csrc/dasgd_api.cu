@@ -34,6 +34,9 @@ struct Slot {
   // last snapshot of this slot recorded.
   std::vector<cudaEvent_t> e_snap_c, e_avg_c;
   bool chunked = false;
+  // Momentum averaging, chunked iterations only: "copy of the buffers written" (main stream) and "mean of the
+  // buffers written" (side stream).  Elsewhere e_snap / e_avg cover the buffers as well.
+  cudaEvent_t e_msnap = nullptr, e_mavg = nullptr;
 };
 
 // A pair of timing events, tagged with what the time between them measures.  For the four kinds of
@@ -113,6 +116,9 @@ struct dasgd_ctx {
   dasgd::DynArgs *dyn_dev = nullptr;
   std::vector<GraphEntry> graphs;
   std::vector<cudaEvent_t> cap_ev;  // per column range, then one per extra lane, then fork and side-stream join
+  // Momentum averaging (dasgd_set_momentum_averaging): copies of the momentum buffers per slot and their means.
+  float *m_snap = nullptr;  // [n_slots][K][ld]
+  float *m_mean = nullptr;  // [n_slots][ld]
   // Sharded worker axis: this context holds cfg.K of K_total workers; `exchange` adds the partial sums of
   // all shards (an all-reduce) on the side stream.  0 / NULL: every worker is here.
   int32_t K_total = 0;
@@ -404,6 +410,25 @@ dasgd_status launch_mean(dasgd_ctx *c, Params p) {
   return st;
 }
 
+float *m_snap_ptr(const dasgd_ctx *c, int slot) { return c->m_snap + (size_t)slot * c->cfg.K * c->cfg.ld; }
+float *m_mean_ptr(const dasgd_ctx *c, int slot) { return c->m_mean + (size_t)slot * c->cfg.ld; }
+
+// Momentum averaging, step 1: the buffers as they are now, copied into the slot's array (main stream).
+dasgd_status copy_momentum(dasgd_ctx *c, int slot) {
+  Params p = base_params(c);
+  p.w = p.m;
+  p.snap_out = m_snap_ptr(c, slot);
+  return launch_snapshot(c, p);
+}
+
+// Step 2: their worker-axis mean (side stream; the caller has ordered the side stream after the copy).
+dasgd_status mean_momentum(dasgd_ctx *c, int slot) {
+  Params p = base_params(c);
+  p.snap_in = m_snap_ptr(c, slot);
+  p.mean_out = m_mean_ptr(c, slot);
+  return launch_mean(c, p);
+}
+
 template <bool BF16, int MODE, bool SNAP>
 dasgd_status launch_merge_t(dasgd_ctx *c, const Params &p) {
   constexpr int EPU = BF16 ? 8 : 4;
@@ -426,8 +451,8 @@ dasgd_status launch_merge_t(dasgd_ctx *c, const Params &p) {
   return DASGD_OK;
 }
 
-dasgd_status launch_merge(dasgd_ctx *c, const Params &p, bool snap) {
-  const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32;
+dasgd_status launch_merge(dasgd_ctx *c, const Params &p, bool snap, bool plain_f32 = false) {
+  const bool bf16 = c->cfg.dtype == DASGD_BF16_MASTER_F32 && !plain_f32;
   const bool delta = c->cfg.merge_mode == DASGD_MERGE_DELTA;
   if (bf16) {
     if (delta) return snap ? launch_merge_t<true, 2, true>(c, p) : launch_merge_t<true, 2, false>(c, p);
@@ -510,6 +535,10 @@ int pick_w_out(const dasgd_ctx *c, int reusable) {
 // book-keeping after the main stream has been given the work that completes the snapshot in pool[buf]
 dasgd_status mark_snapped(dasgd_ctx *c, int slot, int buf) {
   Slot &sl = c->slots[slot];
+  if (c->m_snap) {
+    dasgd_status st = copy_momentum(c, slot);
+    if (st != DASGD_OK) return st;
+  }
   CU(c, cudaEventRecord(sl.e_snap, c->s0));
   sl.state = SLOT_SNAPPED;
   sl.chunked = false;
@@ -546,6 +575,21 @@ dasgd_status wait_oldest_average(dasgd_ctx *c, int *slot_out) {
   return DASGD_OK;
 }
 
+// Momentum averaging, step 3: blend the slot's mean of the buffers into the buffers, on the main stream, after
+// the kernels of this iteration that update them.  The same blend as for the weights; no bfloat16 copy exists.
+dasgd_status merge_momentum(dasgd_ctx *c, int slot) {
+  if (!c->m_snap) return DASGD_OK;
+  Slot &sl = c->slots[slot];
+  if (sl.chunked) CU(c, cudaStreamWaitEvent(c->s0, sl.e_mavg, 0));  // otherwise e_avg, already waited for, covers it
+  Params p = base_params(c);
+  p.w = p.m;
+  p.w_out = p.m;
+  p.w_lp = nullptr;
+  p.mean = m_mean_ptr(c, slot);
+  p.snap_in = m_snap_ptr(c, slot);
+  return launch_merge(c, p, false, true);
+}
+
 void release_oldest(dasgd_ctx *c) {
   const int slot = c->pending.front();
   c->pending.pop_front();
@@ -562,7 +606,9 @@ void destroy_slot_events(Slot &sl) {
   if (sl.e_avg) cudaEventDestroy(sl.e_avg);
   for (cudaEvent_t e : sl.e_snap_c) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : sl.e_avg_c) if (e) cudaEventDestroy(e);
-  sl.e_snap = sl.e_avg = nullptr;
+  if (sl.e_msnap) cudaEventDestroy(sl.e_msnap);
+  if (sl.e_mavg) cudaEventDestroy(sl.e_mavg);
+  sl.e_snap = sl.e_avg = sl.e_msnap = sl.e_mavg = nullptr;
   sl.e_snap_c.clear();
   sl.e_avg_c.clear();
 }
@@ -586,6 +632,10 @@ dasgd_status do_average(dasgd_ctx *c) {
   p.mean_out = mean_ptr(c, slot);
   dasgd_status st = launch_mean(c, p);
   if (st != DASGD_OK) return st;
+  if (c->m_snap) {
+    st = mean_momentum(c, slot);
+    if (st != DASGD_OK) return st;
+  }
   CU(c, cudaEventRecord(sl.e_avg, c->s1));
   sl.stall_sp = stall_mean_done(c, sl.stall_sp);
   sl.state = SLOT_AVERAGING;
@@ -1051,7 +1101,7 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
   // The mean of a range reads the weights its step kernel has just written: store them with the default
   // cache policy so that part of them is still in L2 then (everything else streams through).
   p.keep_w = s_due ? 1 : 0;
-  if (c->use_graph && !(c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0) {
+  if (c->use_graph && !(c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0 && !c->m_snap) {
     dasgd_status gst = replay_chunked(c, p, q, grads, lr, mode, vec, m_due, s_due, per_chunk_wait, ms);
     if (gst != DASGD_OK) return gst;
     if (c->use_graph) {  // replayed (a failed capture switches replay off and falls through to direct launches)
@@ -1115,7 +1165,7 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
       }
     }
   }
-  if (c->use_graph && (c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0 && s_due) {
+  if (c->use_graph && (c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0 && !c->m_snap && s_due) {
     // Timing pass of the replayed schedule: a replay ends only when its last mean is complete, so the
     // main stream waits for it here as well (and that wait is accounted as stall like any other).
     Slot &sl = c->slots[ns];
@@ -1125,6 +1175,22 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
   for (size_t j = 0; j < c->lanes.size(); ++j) {  // join: what the caller puts on the main stream next comes after all lanes
     CU(c, cudaEventRecord(c->e_joins[j], c->lanes[j]));
     CU(c, cudaStreamWaitEvent(c->s0, c->e_joins[j], 0));
+  }
+  if (c->m_snap) {  // momentum averaging: whole-array kernels after the ranges, merge before snapshot as for the weights
+    if (m_due) {
+      dasgd_status st = merge_momentum(c, ms);
+      if (st != DASGD_OK) return st;
+    }
+    if (s_due) {
+      Slot &sl = c->slots[ns];
+      dasgd_status st = copy_momentum(c, ns);
+      if (st != DASGD_OK) return st;
+      CU(c, cudaEventRecord(sl.e_msnap, c->s0));
+      CU(c, cudaStreamWaitEvent(c->s1, sl.e_msnap, 0));
+      st = mean_momentum(c, ns);
+      if (st != DASGD_OK) return st;
+      CU(c, cudaEventRecord(sl.e_mavg, c->s1));
+    }
   }
   c->cur = out;
   c->t += 1;
@@ -1171,6 +1237,8 @@ dasgd_status dasgd_merge(dasgd_ctx *ctx) {
   if (st != DASGD_OK) return st;
   st = op_merge(ctx, slot, -1);
   if (st != DASGD_OK) return st;
+  st = merge_momentum(ctx, slot);
+  if (st != DASGD_OK) return st;
   release_oldest(ctx);
   return DASGD_OK;
 }
@@ -1206,7 +1274,11 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
   }
   st = op_step(ctx, grads, lr, merge_slot, stored_in);
   if (st != DASGD_OK) return st;
-  if (fuse_merge) release_oldest(ctx);
+  if (fuse_merge) {
+    st = merge_momentum(ctx, merge_slot);
+    if (st != DASGD_OK) return st;
+    release_oldest(ctx);
+  }
 
   // ---- separate merge kernel (d == 1, or fusion off), optionally storing the snapshot
   if (m_due && !fuse_merge) {
@@ -1217,6 +1289,8 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
       if (stored_in < 0) return fail(ctx, DASGD_ERR_NO_SLOT, "step: no free snapshot array");
     }
     st = op_merge(ctx, merge_slot, stored_in);
+    if (st != DASGD_OK) return st;
+    st = merge_momentum(ctx, merge_slot);
     if (st != DASGD_OK) return st;
     release_oldest(ctx);
   }
@@ -1232,6 +1306,8 @@ dasgd_status dasgd_step(dasgd_ctx *ctx, const void *grads, float lr) {
       st = wait_oldest_average(ctx, &slot);
       if (st != DASGD_OK) return st;
       st = op_merge(ctx, slot, -1);
+      if (st != DASGD_OK) return st;
+      st = merge_momentum(ctx, slot);
       if (st != DASGD_OK) return st;
       release_oldest(ctx);
     }
@@ -1500,11 +1576,56 @@ dasgd_status dasgd_set_shard(dasgd_ctx *ctx, int32_t K_total, dasgd_exchange_fn 
     return fail(ctx, DASGD_ERR_INVALID_ARG, "set_shard: need K_total >= K and an exchange function");
   if (ctx->cfg.flags & DASGD_FLAG_INLINE_MEAN)
     return fail(ctx, DASGD_ERR_UNSUPPORTED, "set_shard: the inline-mean schedule keeps every worker in one context");
+  if (ctx->m_snap) return fail(ctx, DASGD_ERR_UNSUPPORTED, "set_shard: not available together with momentum averaging");
   if (ctx->t != 0 || !ctx->pending.empty())
     return fail(ctx, DASGD_ERR_BAD_STATE, "set_shard: the context has already been used");
   ctx->K_total = K_total;
   ctx->exchange = exchange;
   ctx->exchange_user = user;
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_set_momentum_averaging(dasgd_ctx *ctx, void *m_snap, void *m_mean) {
+  if (!ctx) return DASGD_ERR_INVALID_ARG;
+  if (!m_snap || !m_mean || !aligned16(m_snap) || !aligned16(m_mean))
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "set_momentum_averaging: m_snap and m_mean must be 16-byte aligned device arrays");
+  if (ctx->cfg.momentum == 0.0f || !ctx->cfg.m)
+    return fail(ctx, DASGD_ERR_INVALID_ARG, "set_momentum_averaging: the context has no momentum buffers");
+  if (ctx->cfg.flags & DASGD_FLAG_INLINE_MEAN)
+    return fail(ctx, DASGD_ERR_UNSUPPORTED, "set_momentum_averaging: not available with DASGD_FLAG_INLINE_MEAN");
+  if (ctx->K_total > 0) return fail(ctx, DASGD_ERR_UNSUPPORTED, "set_momentum_averaging: not available on a sharded worker axis");
+  if (ctx->t != 0 || !ctx->pending.empty())
+    return fail(ctx, DASGD_ERR_BAD_STATE, "set_momentum_averaging: the context has already been used");
+  DeviceGuard guard(ctx->cfg.device);
+  for (void *p : {m_snap, m_mean}) {
+    cudaPointerAttributes at{};
+    cudaError_t e = cudaPointerGetAttributes(&at, p);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return cuda_fail(ctx, e, "set_momentum_averaging: cudaPointerGetAttributes");
+    }
+    if ((at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) ||
+        (at.type == cudaMemoryTypeDevice && at.device != ctx->cfg.device))
+      return fail(ctx, DASGD_ERR_INVALID_ARG, "set_momentum_averaging: m_snap and m_mean must be device memory of cfg.device");
+  }
+  for (Slot &sl : ctx->slots) {
+    if (sl.e_msnap) continue;
+    if (cudaEventCreateWithFlags(&sl.e_msnap, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&sl.e_mavg, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, DASGD_ERR_CUDA, "set_momentum_averaging: cannot create events");
+    }
+  }
+  ctx->m_snap = static_cast<float *>(m_snap);
+  ctx->m_mean = static_cast<float *>(m_mean);
+  return DASGD_OK;
+}
+
+dasgd_status dasgd_get_pending_momentum(const dasgd_ctx *ctx, int32_t i, void **m_snap_device, void **m_mean_device) {
+  if (!ctx || !ctx->m_snap || i < 0 || i >= (int32_t)ctx->pending.size()) return DASGD_ERR_INVALID_ARG;
+  const int slot = ctx->pending[i];
+  if (m_snap_device) *m_snap_device = m_snap_ptr(ctx, slot);
+  if (m_mean_device) *m_mean_device = m_mean_ptr(ctx, slot);
   return DASGD_OK;
 }
 
