@@ -75,7 +75,8 @@ def schedule_of(wl, args):
         return {"merge": "separate", "n_chunks": 0, "lanes": 0, "copy_snapshot": True}
     if wl["d"] >= 1 and args.chunks != 1 and wl["P"] >= 2 * 4096:
         n = args.chunks if args.chunks > 0 else auto_chunks(wl["K"], wl["P"])
-        return {"merge": "chunked", "n_chunks": n, "lanes": 1 if args.lanes else 0, "graph": 1 if args.graph else 0}
+        return {"merge": "chunked", "n_chunks": n, "lanes": 1 if args.lanes else 0, "graph": 1 if args.graph else 0,
+                "side_streams": 2 if args.sides == 2 and wl["K"] >= 4 else 1}   # K = 2: one side stream measured 2 % faster
     if wl["d"] >= 2:
         return {"merge": "fused", "n_chunks": 0, "lanes": 0}
     return {"merge": "separate", "n_chunks": 0, "lanes": 0}
@@ -347,6 +348,8 @@ class Bench:
             f |= B.DASGD_FLAG_TWO_LANES
         if sched.get("graph"):
             f |= B.DASGD_FLAG_GRAPH
+        if sched.get("side_streams") == 2:
+            f |= B.DASGD_FLAG_TWO_SIDE_STREAMS
         return f | (B.DASGD_FLAG_TIMING if timing else 0)
 
     def make(self, wl, sched, timing=False, host_staging=False, flags=None, snapshot_arrays=True):
@@ -699,7 +702,7 @@ def mlp_figures(args):
     base = B.DASGD_FLAG_ROTATE_SNAPSHOT | B.DASGD_FLAG_FUSE_MERGE | B.DASGD_FLAG_TIMING
     n_chunks = auto_chunks(K, P)
     variants = (("separate_merge", base, 0), ("merge_in_step_kernel", base | B.DASGD_FLAG_FUSE_MERGE_D1, 0),
-                ("chunked_pipeline", base | B.DASGD_FLAG_TWO_LANES, n_chunks),
+                ("chunked_pipeline", base | B.DASGD_FLAG_TWO_LANES | B.DASGD_FLAG_TWO_SIDE_STREAMS, n_chunks),
                 ("inline_mean", B.DASGD_FLAG_INLINE_MEAN | B.DASGD_FLAG_TIMING, 0))
     out = {"P": P, "n_chunks": n_chunks}
     for name, flags, chunks in variants:
@@ -798,6 +801,7 @@ def main():
                     help="initialise the NCCL process group even with one rank (exercises the multi-rank plumbing)")
     ap.add_argument("--no-ablation", action="store_true", help="skip the inline-mean ablation leg")
     ap.add_argument("--lanes", type=int, default=1, help="1: alternate the column ranges between two streams; 0: one stream")
+    ap.add_argument("--sides", type=int, default=2, help="2: the means of odd column ranges run on a second side stream; 1: one side stream")
     ap.add_argument("--graph", type=int, default=0, help="1: replay each chunked iteration from a CUDA graph")
     ap.add_argument("--chunks", type=int, default=0,
                     help="column ranges of the pipeline (merge folded into the step kernel); 0: by size "

@@ -106,6 +106,14 @@ typedef enum {
                                          Ignored with DASGD_FLAG_TIMING (which times the same dependency structure
                                          with direct launches) and with a sharded worker axis.  Results unchanged. */
 
+#define DASGD_FLAG_TWO_SIDE_STREAMS 0x400u /* with n_chunks > 1: the means of odd column ranges run on a second side
+                                         stream owned by the library (same priority as side_stream), so that the mean
+                                         of one range does not queue behind the mean of the range before it.  The two
+                                         meet again at the end of every group of ranges and at the end of the
+                                         dasgd_step call: whatever the caller orders after side_stream still comes
+                                         after all means.  The best number of ranges becomes much less critical.
+                                         Has no effect on a sharded worker axis.  Results unchanged.              */
+
 /* Variants of the local step.  Section IV-A states only the values of momentum and weight decay used on the
  * paper's platform and gives no formula, so the common forms are all offered; the default is the plain one. */
 #define DASGD_FLAG_NESTEROV 0x20u      /* w <- w - lr*(g' + mu*m) with the freshly updated m (needs momentum > 0) */

@@ -29,6 +29,7 @@ DASGD_FLAG_NESTEROV, DASGD_FLAG_DECOUPLED_WD = 0x20, 0x40
 DASGD_FLAG_FUSE_MERGE_D1 = 0x80
 DASGD_FLAG_TWO_LANES = 0x100
 DASGD_FLAG_GRAPH = 0x200
+DASGD_FLAG_TWO_SIDE_STREAMS = 0x400
 
 EXPORTS = [
     "dasgd_init", "dasgd_local_step", "dasgd_snapshot", "dasgd_average_async", "dasgd_merge", "dasgd_sync",

@@ -107,6 +107,11 @@ struct dasgd_ctx {
   // DASGD_FLAG_TWO_LANES: odd column ranges run on this stream, forked from and joined to the main
   // stream inside every chunked iteration, so that the kernel of range i+1 fills the SMs as the kernel
   // of range i drains instead of waiting for the stream's next command.
+  // DASGD_FLAG_TWO_SIDE_STREAMS: the means of odd column ranges run on this stream (same priority as the side
+  // stream), so that the mean of range i+1 need not wait for the mean of range i; e_cross orders one side stream
+  // after the other where the two have to meet (end of a group of ranges, end of the iteration).
+  cudaStream_t s1b = nullptr;
+  cudaEvent_t e_cross = nullptr;
   std::vector<cudaStream_t> lanes;      // extra lanes (lane 0 is the main stream)
   std::vector<cudaEvent_t> e_joins;     // one per extra lane
   cudaEvent_t e_fork = nullptr;
@@ -269,12 +274,12 @@ void span_end(dasgd_ctx *c, int idx, cudaStream_t stream) { span_record(c, idx, 
 
 // Stall accounting.  mean_done: called right after a mean kernel has been put on the side stream; the
 // returned span is kept in the slot.  about_to_wait: called where `stream` is about to wait for that mean.
-int stall_mean_done(dasgd_ctx *c, int old_idx) {
+int stall_mean_done(dasgd_ctx *c, int old_idx, cudaStream_t side = nullptr) {
   if (old_idx >= 0 && old_idx < (int)c->spans.size() && c->spans[old_idx].open && c->spans[old_idx].tag == TAG_STALL &&
       !c->spans[old_idx].rec[0])
     c->spans[old_idx].open = false;  // the previous mean of this slot was never waited for
   const int idx = span_alloc(c, TAG_STALL, 0);
-  span_record(c, idx, 1, c->s1);
+  span_record(c, idx, 1, side ? side : c->s1);
   return idx;
 }
 
@@ -361,7 +366,7 @@ dasgd_status launch_snapshot(dasgd_ctx *c, const Params &p) {
   return DASGD_OK;
 }
 
-dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
+dasgd_status launch_reduce(dasgd_ctx *c, const Params &p, cudaStream_t side) {
   long long done = 0;
   if (c->vec) {
     const long long units = p.P / 4;
@@ -369,15 +374,15 @@ dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
       // Shapes chosen by timing each kernel alone on B200 at P = 25.6M (fraction of the measured copy
       // bandwidth): two columns per thread, four rows per batch, three CTAs per SM: 0.97 at K = 8,
       // 1.02 at K = 16, 1.05 at K = 32; all rows in registers for K <= 4: 0.90 (K = 2) to 0.95 (K = 4).
-      if (p.K > 4) dasgd::k_reduce_vec<2, 4, 3><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
-      else if (p.K > 2) dasgd::k_reduce_small<2, 1><<<blocks_for(units, kThreads * 2), kThreads, 0, c->s1>>>(p);
-      else dasgd::k_reduce_small<4, 1><<<blocks_for(units, kThreads * 4), kThreads, 0, c->s1>>>(p);
+      if (p.K > 4) dasgd::k_reduce_vec<2, 4, 3><<<blocks_for(units, kThreads * 2), kThreads, 0, side>>>(p);
+      else if (p.K > 2) dasgd::k_reduce_small<2, 1><<<blocks_for(units, kThreads * 2), kThreads, 0, side>>>(p);
+      else dasgd::k_reduce_small<4, 1><<<blocks_for(units, kThreads * 4), kThreads, 0, side>>>(p);
       c->launches++;
     }
     done = units * 4;
   }
   if (done < p.P) {
-    dasgd::k_reduce_scalar<<<blocks_for(p.P - done, kThreads), kThreads, 0, c->s1>>>(p, done);
+    dasgd::k_reduce_scalar<<<blocks_for(p.P - done, kThreads), kThreads, 0, side>>>(p, done);
     c->launches++;
   }
   CU(c, cudaGetLastError());
@@ -389,24 +394,26 @@ dasgd_status launch_reduce(dasgd_ctx *c, const Params &p) {
 // context's rows (no kernel when there is a single row: the row is its own sum), then the exchange adds
 // the sums of all shards in place; the division by the total number of workers happens where the merge
 // reads the result.
-dasgd_status launch_mean(dasgd_ctx *c, Params p) {
-  const int sp = span_begin(c, TAG_MEAN, c->s1, (long long)p.K * p.P);
+// `side`: the stream it runs on (the caller's side stream unless stated otherwise).
+dasgd_status launch_mean(dasgd_ctx *c, Params p, cudaStream_t side = nullptr) {
+  if (!side) side = c->s1;
+  const int sp = span_begin(c, TAG_MEAN, side, (long long)p.K * p.P);
   dasgd_status st = DASGD_OK;
   if (c->K_total == 0) {
-    st = launch_reduce(c, p);
+    st = launch_reduce(c, p, side);
   } else {
     const float *send = p.snap_in;
     if (p.K > 1) {
       p.sum_only = 1;
-      st = launch_reduce(c, p);
+      st = launch_reduce(c, p, side);
       send = p.mean_out;
     }
     if (st == DASGD_OK) {
-      st = c->exchange(c->exchange_user, send, p.mean_out, p.P, c->s1);
+      st = c->exchange(c->exchange_user, send, p.mean_out, p.P, side);
       if (st != DASGD_OK) fail(c, st, "average: the exchange of the partial sums failed");
     }
   }
-  span_end(c, sp, c->s1);
+  span_end(c, sp, side);
   return st;
 }
 
@@ -790,6 +797,17 @@ dasgd_status dasgd_init(dasgd_ctx **out, const dasgd_config *cfg) {
       return fail(nullptr, DASGD_ERR_CUDA, "init: cannot create the second lane's stream and events");
     }
   }
+  if (ctx->chunks > 1 && (c.flags & DASGD_FLAG_TWO_SIDE_STREAMS)) {
+    int prio = 0;
+    const bool ok = cudaStreamGetPriority(ctx->s1, &prio) == cudaSuccess &&
+                    cudaStreamCreateWithPriority(&ctx->s1b, cudaStreamNonBlocking, prio) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&ctx->e_cross, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      dasgd_destroy(ctx);
+      return fail(nullptr, DASGD_ERR_CUDA, "init: cannot create the second side stream");
+    }
+  }
   if (ctx->chunks > 1 && (c.flags & DASGD_FLAG_GRAPH)) {
     bool ok = cudaMalloc(&ctx->dyn_dev, sizeof(dasgd::DynArgs)) == cudaSuccess;
     const size_t n_ev = (size_t)ctx->chunks + ctx->lanes.size() + 2;
@@ -839,6 +857,11 @@ dasgd_status dasgd_destroy(dasgd_ctx *ctx) {
     cudaStreamSynchronize(st);
     cudaStreamDestroy(st);
   }
+  if (ctx->s1b) {
+    cudaStreamSynchronize(ctx->s1b);
+    cudaStreamDestroy(ctx->s1b);
+  }
+  if (ctx->e_cross) cudaEventDestroy(ctx->e_cross);
   for (cudaEvent_t ev : ctx->e_joins) cudaEventDestroy(ev);
   for (GraphEntry &g : ctx->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
   for (cudaEvent_t ev : ctx->cap_ev) cudaEventDestroy(ev);
@@ -1138,6 +1161,9 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
   // An iteration that only merges (no snapshot follows it) has no mean to feed, so the ranges of a group go
   // out as one launch: the group is the granularity of the waits anyway.
   const int stride = s_due ? 1 : G;
+  // Two side streams only with every worker here: the exchange of a sharded worker axis is a collective, and the
+  // ranks must issue those in one order on one stream.
+  const bool two_sides = c->s1b != nullptr && c->K_total == 0;
   for (int i = 0; i < C; i += stride) {
     const int last = i + stride - 1 < C - 1 ? i + stride - 1 : C - 1;   // last range of this launch
     const long long col0 = (long long)i * c->chunk_cols;
@@ -1155,15 +1181,25 @@ dasgd_status step_chunked(dasgd_ctx *c, const void *grads, float lr, bool m_due,
     if (st != DASGD_OK) return st;
     if (s_due) {
       Slot &sl = c->slots[ns];
+      cudaStream_t side = (two_sides && (i & 1)) ? c->s1b : c->s1;
       CU(c, cudaEventRecord(sl.e_snap_c[i], lane));
-      CU(c, cudaStreamWaitEvent(c->s1, sl.e_snap_c[i], 0));
-      st = launch_mean(c, columns(c, q, col0, len));
+      CU(c, cudaStreamWaitEvent(side, sl.e_snap_c[i], 0));
+      st = launch_mean(c, columns(c, q, col0, len), side);
       if (st != DASGD_OK) return st;
       if (i == group_end(i)) {
-        CU(c, cudaEventRecord(sl.e_avg_c[i], c->s1));
-        sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i]);
+        if (two_sides) {  // "mean of range i complete" must imply the earlier ranges on the other side stream too
+          cudaStream_t other = (i & 1) ? c->s1 : c->s1b;
+          CU(c, cudaEventRecord(c->e_cross, other));
+          CU(c, cudaStreamWaitEvent(side, c->e_cross, 0));
+        }
+        CU(c, cudaEventRecord(sl.e_avg_c[i], side));
+        sl.stall_sp_c[i] = stall_mean_done(c, sl.stall_sp_c[i], side);
       }
     }
+  }
+  if (two_sides && s_due) {  // the caller's side stream again comes after everything this iteration averaged
+    CU(c, cudaEventRecord(c->e_cross, c->s1b));
+    CU(c, cudaStreamWaitEvent(c->s1, c->e_cross, 0));
   }
   if (c->use_graph && (c->cfg.flags & DASGD_FLAG_TIMING) && c->K_total == 0 && !c->m_snap && s_due) {
     // Timing pass of the replayed schedule: a replay ends only when its last mean is complete, so the
@@ -1349,6 +1385,7 @@ dasgd_status dasgd_sync(dasgd_ctx *ctx) {
   DeviceGuard guard(ctx->cfg.device);
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(ctx->cfg.sync_timeout_ms);
   std::vector<cudaStream_t> streams = {ctx->s0, ctx->s1};
+  if (ctx->s1b) streams.push_back(ctx->s1b);
   if (ctx->s_copy) streams.push_back(ctx->s_copy);
   for (cudaStream_t st : ctx->lanes) streams.push_back(st);
   for (cudaStream_t s : streams) {

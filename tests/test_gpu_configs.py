@@ -17,7 +17,7 @@ from paper_2006_00441_b200 import inputs
 from tests.harness import TOL_RUN, TOL_STEP, assert_close, bf16_bits, to_oracle_grad
 
 pytestmark = pytest.mark.gpu
-FUSED = 0x4 | 0x8 | 0x100   # snapshots by array rotation; merge folded into the step kernel; two lanes when chunked
+FUSED = 0x4 | 0x8 | 0x100 | 0x400   # snapshots by array rotation; merge folded into the step kernel; two lanes and two side streams when chunked
 def chunks_for(K, P, d):
     """The benchmark's policy for the number of column ranges."""
     import bench

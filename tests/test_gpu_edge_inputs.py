@@ -10,7 +10,7 @@ from tests.harness import TOL_RUN, TOL_STEP, make_pair, padded_grad, to_oracle_g
 
 pytestmark = pytest.mark.gpu
 FUSE_SNAP, FUSE_MERGE, ROTATE, INLINE, LANES, FUSE_D1 = 0x2, 0x4, 0x8, 0x10, 0x100, 0x80
-SCHEDS = [(0, 0), (ROTATE | FUSE_MERGE | LANES, 3), (ROTATE | FUSE_MERGE | FUSE_D1, 0), (FUSE_SNAP | FUSE_MERGE, 0), (INLINE, 0)]
+SCHEDS = [(0, 0), (ROTATE | FUSE_MERGE | LANES | 0x400, 3), (ROTATE | FUSE_MERGE | FUSE_D1, 0), (FUSE_SNAP | FUSE_MERGE, 0), (INLINE, 0)]
 
 
 @pytest.fixture(scope="module")

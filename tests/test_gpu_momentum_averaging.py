@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 
 FUSE_SNAP, FUSE_MERGE, ROTATE, INLINE, FUSE_D1, LANES, GRAPH = 0x2, 0x4, 0x8, 0x10, 0x80, 0x100, 0x200
 SCHEDS = [(0, 0), (FUSE_SNAP | FUSE_MERGE, 0), (ROTATE, 0), (ROTATE | FUSE_MERGE, 0), (ROTATE | FUSE_MERGE | FUSE_D1, 0),
-          (ROTATE | FUSE_MERGE, 3), (ROTATE | FUSE_MERGE | LANES, 2), (ROTATE | FUSE_MERGE | LANES | GRAPH, 3)]
+          (ROTATE | FUSE_MERGE, 3), (ROTATE | FUSE_MERGE | LANES, 2), (ROTATE | FUSE_MERGE | LANES | GRAPH, 3),
+          (ROTATE | FUSE_MERGE | LANES | 0x400, 3)]
 SCHEDULES = [(1, 1), (2, 1), (1, 2), (2, 2), (3, 2), (2, 3), (3, 0), (1, 0)]
 
 

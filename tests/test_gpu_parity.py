@@ -15,10 +15,11 @@ pytestmark = pytest.mark.gpu
 
 FUSE_SNAP, FUSE_MERGE, ROTATE, INLINE = 0x2, 0x4, 0x8, 0x10
 NESTEROV, DECOUPLED = 0x20, 0x40
-FUSE_D1, LANES, GRAPH = 0x80, 0x100, 0x200
+FUSE_D1, LANES, GRAPH, SIDES = 0x80, 0x100, 0x200, 0x400
 # schedules of dasgd_step: (flags, n_chunks).  The chunked pipeline applies to every d >= 1.
 SCHEDS = [(0, 0), (FUSE_SNAP, 0), (FUSE_MERGE, 0), (FUSE_SNAP | FUSE_MERGE, 0), (ROTATE, 0), (ROTATE | FUSE_MERGE, 0),
           (ROTATE | FUSE_MERGE, 3), (ROTATE | FUSE_MERGE, 2), (ROTATE | FUSE_MERGE | LANES, 3), (ROTATE | FUSE_MERGE | LANES | GRAPH, 3), (ROTATE | FUSE_MERGE | GRAPH, 2),
+          (ROTATE | FUSE_MERGE | LANES | SIDES, 3), (ROTATE | FUSE_MERGE | SIDES, 2),
           (ROTATE | FUSE_MERGE | FUSE_D1, 0), (FUSE_MERGE | FUSE_D1, 0),
           (INLINE, 0)]
 # f32 vector tile = 256 threads * 4 units * 4 elements = 4096 elements; bf16 tile = 256*2*8 = 4096
