@@ -42,7 +42,7 @@ typedef enum {
   DASGD_ERR_NO_SLOT = 3,       /* snapshot requested while every slot holds a pending average */
   DASGD_ERR_CUDA = 4,          /* a CUDA runtime call failed; see dasgd_last_error            */
   DASGD_ERR_TIMEOUT = 5,       /* dasgd_sync gave up waiting                                  */
-  DASGD_ERR_UNSUPPORTED = 6    /* valid request this build cannot serve                       */
+  DASGD_ERR_UNSUPPORTED = 6    /* valid request this library cannot serve                     */
 } dasgd_status;
 
 typedef enum {
