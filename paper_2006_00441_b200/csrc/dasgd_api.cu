@@ -296,8 +296,8 @@ bool fits_one_launch(const Params &p) { return ((p.P + 4095) / 4096) * (long lon
 
 template <bool BF16, bool MOM, int MERGE, bool SNAP>
 dasgd_status launch_step_t(dasgd_ctx *c, const Params &p, bool vec, cudaStream_t stream) {
-  constexpr int EPU = BF16 ? 8 : 4;
-  constexpr int UNROLL = BF16 ? 2 : 4;
+  constexpr int EPU = 4;     // elements per unit of the vector step kernel, both dtypes
+  constexpr int UNROLL = 4;
   long long done = 0;
   if (vec) {
     const long long units = p.P / EPU;

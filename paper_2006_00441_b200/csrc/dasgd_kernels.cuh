@@ -67,6 +67,13 @@ __device__ __forceinline__ void st_stream(float4 *p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(uint4 *p, uint4 v) { __stcs(p, v); }
 
+// 16 bytes from global to shared memory without passing through registers (completion: cp_async_wait_all).
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
 
 // two float32 -> packed bf16x2, round to nearest even (lo in the low half)
@@ -121,8 +128,11 @@ __device__ __forceinline__ float blend_delta(float w, float mean, float snap) {
 
 // ---------------------------------------------------------------- local step (vector path)
 //
-// One CTA = one worker k and one tile of kThreads*UNROLL units; a unit is 4 (float32 gradients) or
-// 8 (bfloat16 gradients) consecutive parameters.  With a fused merge blockIdx.x enumerates (tile, k)
+// One CTA = one worker k and one tile of kThreads*UNROLL units; a unit is 4 consecutive parameters in both
+// dtypes: the float32 arrays are read and written as one 16-byte access per unit, bfloat16 gradients and the
+// bfloat16 weight copy as one 8-byte access per unit, so that every warp-wide access covers a contiguous range
+// (with 8-element units each lane would touch two separate halves of a 32-byte sector of the float32 arrays).
+// With a fused merge blockIdx.x enumerates (tile, k)
 // with k fastest, so that the K CTAs sharing a mean tile are neighbours in launch order and the tile
 // is fetched from HBM once; otherwise rows are walked one after the other (k slowest), which keeps
 // every CTA wave on one contiguous address range (measured 1.2 % faster).
@@ -132,10 +142,8 @@ __device__ __forceinline__ float blend_delta(float w, float mean, float snap) {
 // registers and lose a third of its resident warps, i.e. of its loads in flight.
 template <bool BF16, bool MOM, int MERGE, bool SNAP>
 __global__ void __launch_bounds__(kThreads, 3) k_local_step_vec(const Params p) {
-  constexpr int EPU = BF16 ? 8 : 4;   // elements per unit
-  constexpr int F4 = EPU / 4;          // float4 per unit
-  constexpr int UNROLL = BF16 ? 2 : 4; // units per thread
-  const long long units = p.P / EPU;
+  constexpr int UNROLL = 4;  // units per thread
+  const long long units = p.P / 4;
   int k;
   long long tile;
   if (MERGE != 0) {
@@ -155,68 +163,63 @@ __global__ void __launch_bounds__(kThreads, 3) k_local_step_vec(const Params p) 
     lr = p.dyn->lr;
   }
 
-  float4 w4[UNROLL][F4], m4[UNROLL][F4], g4[UNROLL][F4], a4[UNROLL][F4], s4[UNROLL][F4];
+  float4 w4[UNROLL], m4[UNROLL], g4[UNROLL], s4[UNROLL];
   bool ok[UNROLL];
+  // The piece of the mean this CTA blends with is staged in shared memory by asynchronous copies: it then holds no
+  // registers while in flight (with it in registers the kernel wants 90, and at the 80 that three CTAs per SM
+  // allow the compiler can no longer issue all loads before the first use).  Every thread reads back only what it
+  // copied itself, so waiting for its own copies is enough; no barrier.
+  __shared__ float4 s_mean[MERGE != 0 ? UNROLL : 1][MERGE != 0 ? kThreads : 1];
 
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j) {
     const long long u = u0 + (long long)j * kThreads;
     ok[j] = u < units;
     if (ok[j]) {
-      const long long e = u * EPU;  // element offset inside the row
+      const long long e = u * 4;  // element offset inside the row
       if (BF16) {
-        const uint4 gb = ld_stream(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(gbase) + row + e));
-        g4[j][0] = make_float4(bf16_bits_to_f32(gb.x & 0xFFFFu), bf16_bits_to_f32(gb.x >> 16),
-                               bf16_bits_to_f32(gb.y & 0xFFFFu), bf16_bits_to_f32(gb.y >> 16));
-        g4[j][F4 - 1] = make_float4(bf16_bits_to_f32(gb.z & 0xFFFFu), bf16_bits_to_f32(gb.z >> 16),
-                                    bf16_bits_to_f32(gb.w & 0xFFFFu), bf16_bits_to_f32(gb.w >> 16));
+        const uint2 gb = __ldcs(reinterpret_cast<const uint2 *>(static_cast<const __nv_bfloat16 *>(gbase) + row + e));
+        g4[j] = make_float4(bf16_bits_to_f32(gb.x & 0xFFFFu), bf16_bits_to_f32(gb.x >> 16),
+                            bf16_bits_to_f32(gb.y & 0xFFFFu), bf16_bits_to_f32(gb.y >> 16));
       } else {
-        g4[j][0] = ld_stream(reinterpret_cast<const float4 *>(static_cast<const float *>(gbase) + row + e));
+        g4[j] = ld_stream(reinterpret_cast<const float4 *>(static_cast<const float *>(gbase) + row + e));
       }
-#pragma unroll
-      for (int f = 0; f < F4; ++f) {
-        w4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.w + row + e) + f);
-        if (MOM) m4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.m + row + e) + f);
-        if (MERGE != 0) a4[j][f] = mean_of(__ldg(reinterpret_cast<const float4 *>(p.mean + e) + f), p);
-        if (MERGE == 2) s4[j][f] = ld_stream(reinterpret_cast<const float4 *>(p.snap_in + row + e) + f);
-      }
+      w4[j] = ld_stream(reinterpret_cast<const float4 *>(p.w + row + e));
+      if (MOM) m4[j] = ld_stream(reinterpret_cast<const float4 *>(p.m + row + e));
+      if (MERGE != 0) cp_async16(&s_mean[j][threadIdx.x], p.mean + e);
+      if (MERGE == 2) s4[j] = ld_stream(reinterpret_cast<const float4 *>(p.snap_in + row + e));
     }
   }
 
+  if (MERGE != 0) cp_async_wait_all();
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j) {
     if (!ok[j]) continue;
-    const long long e = (u0 + (long long)j * kThreads) * EPU;
-#pragma unroll
-    for (int f = 0; f < F4; ++f) {
-      float4 w = w4[j][f];
-      float4 m = MOM ? m4[j][f] : make_float4(0.f, 0.f, 0.f, 0.f);
-      const float4 g = g4[j][f];
-      step_elem<MOM>(w.x, m.x, g.x, p, lr);
-      step_elem<MOM>(w.y, m.y, g.y, p, lr);
-      step_elem<MOM>(w.z, m.z, g.z, p, lr);
-      step_elem<MOM>(w.w, m.w, g.w, p, lr);
-      if (MERGE == 1) {
-        const float4 a = a4[j][f];
-        DASGD_F4_APPLY(w, blend_xi(w.x, a.x, p), blend_xi(w.y, a.y, p), blend_xi(w.z, a.z, p), blend_xi(w.w, a.w, p))
-      } else if (MERGE == 2) {
-        const float4 a = a4[j][f], s = s4[j][f];
-        DASGD_F4_APPLY(w, blend_delta(w.x, a.x, s.x), blend_delta(w.y, a.y, s.y), blend_delta(w.z, a.z, s.z),
-                       blend_delta(w.w, a.w, s.w))
-      }
-      if (p.keep_w) reinterpret_cast<float4 *>(p.w_out + row + e)[f] = w;
-      else st_stream(reinterpret_cast<float4 *>(p.w_out + row + e) + f, w);
-      if (MOM) st_stream(reinterpret_cast<float4 *>(p.m + row + e) + f, m);
-      if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + row + e) + f, w);
-      w4[j][f] = w;
+    const long long e = (u0 + (long long)j * kThreads) * 4;
+    float4 w = w4[j];
+    float4 m = MOM ? m4[j] : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 g = g4[j];
+    step_elem<MOM>(w.x, m.x, g.x, p, lr);
+    step_elem<MOM>(w.y, m.y, g.y, p, lr);
+    step_elem<MOM>(w.z, m.z, g.z, p, lr);
+    step_elem<MOM>(w.w, m.w, g.w, p, lr);
+    if (MERGE == 1) {
+      const float4 a = mean_of(s_mean[j][threadIdx.x], p);
+      DASGD_F4_APPLY(w, blend_xi(w.x, a.x, p), blend_xi(w.y, a.y, p), blend_xi(w.z, a.z, p), blend_xi(w.w, a.w, p))
+    } else if (MERGE == 2) {
+      const float4 a = mean_of(s_mean[j][threadIdx.x], p), s = s4[j];
+      DASGD_F4_APPLY(w, blend_delta(w.x, a.x, s.x), blend_delta(w.y, a.y, s.y), blend_delta(w.z, a.z, s.z),
+                     blend_delta(w.w, a.w, s.w))
     }
+    if (p.keep_w) *reinterpret_cast<float4 *>(p.w_out + row + e) = w;
+    else st_stream(reinterpret_cast<float4 *>(p.w_out + row + e), w);
+    if (MOM) st_stream(reinterpret_cast<float4 *>(p.m + row + e), m);
+    if (SNAP) st_stream(reinterpret_cast<float4 *>(p.snap_out + row + e), w);
     if (BF16) {
-      uint4 o;
-      o.x = pack_bf16x2(w4[j][0].x, w4[j][0].y);
-      o.y = pack_bf16x2(w4[j][0].z, w4[j][0].w);
-      o.z = pack_bf16x2(w4[j][F4 - 1].x, w4[j][F4 - 1].y);
-      o.w = pack_bf16x2(w4[j][F4 - 1].z, w4[j][F4 - 1].w);
-      st_stream(reinterpret_cast<uint4 *>(p.w_lp + row + e), o);
+      uint2 o;
+      o.x = pack_bf16x2(w.x, w.y);
+      o.y = pack_bf16x2(w.z, w.w);
+      __stcs(reinterpret_cast<uint2 *>(p.w_lp + row + e), o);
     }
   }
 }
