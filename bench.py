@@ -101,7 +101,7 @@ def path_bytes_per_update(wl, sched):
 # on one column range of the pipeline.  Reads grow with the updates of a launch; the stores that are still
 # dirty in L2 when the kernel ends are a constant, not a share.  Valid only while the kernel source is the
 # one that was profiled.
-NCU_TRAFFIC = {"kernels_sha256_prefix": "7280e949149ba7eb", "updates": 5_275_648, "read_bytes": 65.961e6, "write_bytes": 2.46e6,
+NCU_TRAFFIC = {"kernels_sha256_prefix": "b183982c22bc7811", "updates": 5_275_648, "read_bytes": 65.962e6, "write_bytes": 2.38e6,
                "applies_to": "float32 + momentum, merge folded in"}
 
 
