@@ -101,7 +101,7 @@ def path_bytes_per_update(wl, sched):
 # on one column range of the pipeline.  Reads grow with the updates of a launch; the stores that are still
 # dirty in L2 when the kernel ends are a constant, not a share.  Valid only while the kernel source is the
 # one that was profiled.
-NCU_TRAFFIC = {"kernels_sha256_prefix": "b183982c22bc7811", "updates": 5_275_648, "read_bytes": 65.962e6, "write_bytes": 2.38e6,
+NCU_TRAFFIC = {"kernels_sha256_prefix": "ae8627e365d3f6a1", "updates": 5_275_648, "read_bytes": 65.965e6, "write_bytes": 2.40e6,
                "applies_to": "float32 + momentum, merge folded in"}
 
 

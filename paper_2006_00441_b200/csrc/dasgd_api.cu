@@ -186,6 +186,7 @@ Params base_params(const dasgd_ctx *c) {
   p.xi = c->cfg.xi;
   p.omx = 1.0f - c->cfg.xi;
   p.mean_div = c->K_total > 0 ? (float)c->K_total : 0.0f;
+  p.group_tiles = 1;
   return p;
 }
 
@@ -888,6 +889,11 @@ dasgd_status op_step(dasgd_ctx *c, const void *grads, float lr, int merge_slot, 
     p.mean = mean_ptr(c, merge_slot);
     p.snap_in = snap_ptr(c, merge_slot);
     reusable = reusable_buf(c, merge_slot);
+    // One launch over the whole array: walk the rows in runs of 512 tiles (8 MB per array), so that the CTAs in
+    // flight stream a few long runs instead of K times as many short ones, while the 8 MB of the mean a group
+    // blends with stay in L2 for its K passes.  Measured alone, float32: 6.60 -> 6.78 TB/s at K = 8, 6.65 -> 6.90
+    // at K = 32; groups of 128 or 2048 tiles gain less or nothing.  (Column ranges of the pipeline keep 1.)
+    p.group_tiles = 512;
   }
   const int out = pick_w_out(c, reusable);
   if (out < 0) return fail(c, DASGD_ERR_NO_SLOT, "step: no free weight array to write into");

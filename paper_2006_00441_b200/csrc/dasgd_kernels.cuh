@@ -56,6 +56,7 @@ struct Params {
   float mean_div;    // 0: `mean` holds the mean.  Otherwise `mean` holds the SUM over all workers (sharded
                      //    worker axis) and the mean is that sum divided, correctly rounded, by this number
   int sum_only;      // 1: the worker-axis kernel writes the plain sum of its K rows, not their mean
+  int group_tiles;   // merging step kernel: tiles per group in the CTA order (1: the K rows of a tile are neighbours)
   int keep_w;        // 1: the new weights are about to be re-read (by the mean of this column range): store
                      //    them with the default cache policy instead of the streaming one
 };
@@ -132,10 +133,11 @@ __device__ __forceinline__ float blend_delta(float w, float mean, float snap) {
 // dtypes: the float32 arrays are read and written as one 16-byte access per unit, bfloat16 gradients and the
 // bfloat16 weight copy as one 8-byte access per unit, so that every warp-wide access covers a contiguous range
 // (with 8-element units each lane would touch two separate halves of a 32-byte sector of the float32 arrays).
-// With a fused merge blockIdx.x enumerates (tile, k)
-// with k fastest, so that the K CTAs sharing a mean tile are neighbours in launch order and the tile
-// is fetched from HBM once; otherwise rows are walked one after the other (k slowest), which keeps
-// every CTA wave on one contiguous address range (measured 1.2 % faster).
+// With a fused merge blockIdx.x enumerates groups of group_tiles tiles and, inside a group, (k, tile) with the
+// tile fastest: the K passes over a group re-read the same piece of the mean, which is fetched from HBM once and
+// then served by L2 (group_tiles = 1: the K CTAs of a tile are neighbours in launch order).  Without a merge rows
+// are walked one after the other (k slowest), which keeps every CTA wave on one contiguous address range
+// (measured 1.2 % faster).
 // MERGE: 0 none, 1 xi-blend, 2 delta.  SNAP: also store the final w into snap_out.
 
 // Three CTAs per SM (at most 80 registers): with a merge folded in the kernel would otherwise take 85-96
@@ -147,8 +149,16 @@ __global__ void __launch_bounds__(kThreads, 3) k_local_step_vec(const Params p) 
   int k;
   long long tile;
   if (MERGE != 0) {
-    k = blockIdx.x % p.K;
-    tile = blockIdx.x / p.K;
+    // groups of group_tiles tiles: inside a group the rows are walked one after the other, so that every row is
+    // read and written in contiguous runs while the K CTAs that share a piece of the mean stay close in time
+    const long long tiles = (units + kThreads * UNROLL - 1) / (kThreads * UNROLL);
+    const long long per_group = (long long)p.group_tiles * p.K;
+    const long long grp = blockIdx.x / per_group;
+    const long long r = blockIdx.x - grp * per_group;
+    const long long left = tiles - grp * p.group_tiles;
+    const long long g_eff = left < p.group_tiles ? left : p.group_tiles;
+    k = (int)(r / g_eff);
+    tile = grp * p.group_tiles + r % g_eff;
   } else {
     const unsigned tiles = (unsigned)((units + kThreads * UNROLL - 1) / (kThreads * UNROLL));
     k = blockIdx.x / tiles;

@@ -254,6 +254,26 @@ def test_chunked_pipeline_mixes_with_the_explicit_calls(B, mode):
     assert_close(w, cpu.w, TOL_RUN, "w"); assert_close(m, cpu.m, TOL_RUN, "m")
 
 
+@pytest.mark.parametrize("K,dtype,mode,tau,d", [(3, 0, 0, 1, 1), (2, 1, 0, 1, 2), (5, 0, 1, 2, 2), (4, 1, 1, 1, 1)])
+def test_whole_array_merging_launch_with_several_tile_groups(B, K, dtype, mode, tau, d):
+    """A merge folded into one launch over the whole array walks the rows in groups of 512 tiles of 4096 columns.
+    Here: one full group, a ragged second group (300 tiles and a partial one) and a scalar tail."""
+    P, T = (512 + 300) * 4096 + 1000 + 13, 8
+    ld = (P + 7) // 8 * 8
+    w0 = inputs.shared_start(95, P, 0.02).numpy()
+    gpu, cpu = make_pair(B, K, P, tau, d, 0.25, 0.9, 1e-4, dtype=dtype, merge_mode=mode,
+                         flags=ROTATE | FUSE_MERGE | FUSE_D1, ld=ld, w0=w0)
+    gd = torch.bfloat16 if dtype else torch.float32
+    ring = [grads(96, t, K, P, 0.0316, gd, ld) for t in range(2)]
+    for t in range(T):
+        gpu.step(ring[t % 2], 0.1)
+        cpu.step(to_oracle_grad(ring[t % 2], P), 0.1)
+    w, m = state_of(gpu)
+    assert_close(w, cpu.w, TOL_RUN, "w"); assert_close(m, cpu.m, TOL_RUN, "m")
+    if dtype:
+        np.testing.assert_array_equal(bf16_bits(gpu.w_lp[:, :P]), bf16_bits(gpu.w[:, :P].to(torch.bfloat16)))
+
+
 def test_chunks_need_rotation_fused_merge_and_a_delay(B):
     for kw in (dict(flags=ROTATE), dict(flags=FUSE_MERGE), dict(flags=ROTATE | FUSE_MERGE, d=0), dict(flags=ROTATE | FUSE_MERGE, n_chunks=1025)):
         args = dict(K=2, P=64, tau=2, d=1, xi=0.25, n_chunks=4)
