@@ -136,7 +136,7 @@ def measured_peak_gbs():
 # ------------------------------------------------------------------ clocks
 
 class ClockSampler:
-    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
@@ -153,7 +153,10 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, window=None):
+        """Median SM clock and the throttle reasons seen.  `window` = (t0, t1) in time.time() seconds: only the
+        samples taken inside it count (the sampler is started well before, because nvidia-smi needs a moment to
+        come up); if none falls inside, all samples do, and the summary says so."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
         if self.proc is None:
             return out
@@ -162,28 +165,30 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
-                if len(f) < 7:
+                if len(f) < 8:
                     continue
                 try:
-                    sm.append(float(f[0])); mx.append(float(f[1]))
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(f[1]), float(f[2]), [nm for nm, v in zip(names, f[4:8]) if v.lower().startswith("active")]))
                 except ValueError:
                     continue
-                for nm, v in zip(names, f[3:7]):
-                    if v.lower().startswith("active"):
-                        reasons.add(nm)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out["sm_mhz"] = statistics.median(sm)
-            out["sm_max_mhz"] = max(mx)
-        out["reasons"] = sorted(reasons)
-        out["samples"] = len(sm)
+        inside = [r for r in rows if window and window[0] <= r[0] <= window[1]]
+        used = inside or rows
+        if used:
+            out["sm_mhz"] = statistics.median(r[1] for r in used)
+            out["sm_max_mhz"] = max(r[2] for r in used)
+        out["reasons"] = sorted({nm for r in used for nm in r[3]})
+        out["samples"] = len(used)
+        out["window"] = "timed region" if inside else "whole measurement (no sample fell inside the timed region)"
         return out
 
 
@@ -406,7 +411,9 @@ def measure_workload(bench, wl, sched, steps, warmup, repeats, ring, lr, with_al
 
     out = {}
     eng = bench.make(wl, sched)
+    t_begin = time.time()
     out["headline"] = bench.repeated(eng, steps, warmup, repeats, dev_step)
+    out["headline_window"] = (t_begin, time.time())     # host clock, for the clock sampler: warm-up + the timed loops
     eng.close()
     del eng
 
@@ -499,6 +506,7 @@ def run_ours(args, wl, name, bench=None, compact=False):
     gdt = torch.bfloat16 if bf16 else torch.float32
     RING = wl.get("ring", 4)
     sched = schedule_of(wl, args)
+    sampler = ClockSampler(bench.local_rank) if rank == 0 and not compact else None   # started early: it takes a moment to come up
     seed = 1000 + rank  # every rank runs its own replica of the workload
     ring = [inputs.grad_block(seed, t, K, P, wl["g_std"], device="cuda", dtype=gdt) for t in range(RING)]
     torch.cuda.synchronize()
@@ -508,10 +516,9 @@ def run_ours(args, wl, name, bench=None, compact=False):
 
     if sched["merge"] == "chunked" and args.chunks == 0 and bench.comm is None and not args.no_calibrate:
         sched = calibrate_chunks(bench, wl, sched, ring, lr)
-    sampler = ClockSampler(bench.local_rank) if rank == 0 and not compact else None
     m = measure_workload(bench, wl, sched, args.steps, args.warmup, args.repeats, ring, lr,
                          with_alone=(not compact) or args.sweep)
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(m.get("headline_window")) if sampler else None
     ms = m["headline"]["ms_per_step"]
     value = world * K * P / (ms * 1e-3)
     bpu = path_bytes_per_update(wl, sched)
